@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the batched inverse-Helmholtz tensor-product operator on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload i] [--no-cpu-baseline] [--no-e2e]
+
+One *step* is one pass of the whole operator over the workload's E elements (one
+library call).  Default workload: the largest inverse-Helmholtz configuration
+(n = 14, E = 131072, fp64, 8.63 GB of u/D/v per step -- far larger than L2, so every
+step streams from HBM).  Prints ONE JSON line on rank 0.
+
+For N > 1 launch with ``python -m torch.distributed.run --nproc-per-node N``: every
+rank holds its own E elements (weak scaling; elements are independent, so there is
+no data-path collective -- NCCL is used only for the barrier and the max-over-ranks
+of the device time).
+
+``--impl reference`` times the CPU oracle, as it stands, on the host cores over a
+bounded sample of the same workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "elements/s (fp64 SEM inverse-Helmholtz); GFLOP/s and roofline fraction alongside"
+UNIT = "elements/s"
+
+# FP64 roof derived from unit counts and clocks: 148 SMs x 64 FP64 FMA lanes per SM per
+# clock x 2 flops x 1.965 GHz (clocks.max.sm).
+FP64_LANES_PER_SM = 64
+SM_COUNT = 148
+SM_MAX_GHZ = 1.965
+FP64_PEAK_TFLOPS = SM_COUNT * FP64_LANES_PER_SM * 2 * SM_MAX_GHZ / 1e3
+HBM_FALLBACK_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                return json.load(f), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": HBM_FALLBACK_GBS}, "fallback"
+
+
+# ------------------------------------------------------------------------------ clocks
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML (read-only)."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, uuid: str | None, index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.period = period
+        self.samples, self.power, self.mask = [], [], 0
+        self.sm_max = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-")
+                                                          else "GPU-" + uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self) -> dict:
+        self._halt.set()
+        if self.is_alive():
+            self.join()
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["unavailable"]}
+        reasons = [name for bit, name in self.REASONS.items() if self.mask & bit]
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.sm_max,
+                "sm_min_mhz": min(self.samples), "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None,
+                "reasons": reasons}
+
+
+# ------------------------------------------------------------------------------ CPU oracle leg
+
+def oracle_run(wl, e0, e1):
+    """Oracle over elements [e0,e1) of the workload; returns (seconds, output, inputs)."""
+    import oracle
+    from paper_2604_19906_b200 import inputs
+    host = inputs.host_case(wl, e0, e1)
+    t0 = time.perf_counter()
+    if wl.op == "inv_helmholtz":
+        v = oracle.inv_helmholtz(host["S"], host["D"], host["u"])
+    else:
+        v = oracle.tpo_apply(host["A"], host["B"], host["C"], host["u"])
+    return time.perf_counter() - t0, v, host
+
+
+def cpu_baseline(wl, target_seconds=12.0, max_elements=None):
+    """The oracle, as it stands, on all host cores over a bounded sample (the first Ns
+    elements) of the workload.  Returns the cpu_baseline object, the sample's output."""
+    import oracle
+    probe = min(wl.E, 256)
+    t_probe, _, _ = oracle_run(wl, 0, probe)
+    rate = probe / max(t_probe, 1e-6)
+    ns = int(min(wl.E, max(probe, rate * target_seconds)))
+    if max_elements:
+        ns = min(ns, max_elements)
+    t, v, _ = oracle_run(wl, 0, ns)
+    cores = oracle.threads_used(0)
+    return {"value": ns / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "gflops": ns * wl.flops_per_element / t / 1e9,
+            "sample": f"first {ns} of {wl.E} elements of {wl.name}, {t:.2f} s on {cores} threads"
+            }, v, ns
+
+
+def reference_arm(args, wl, rank):
+    """``--impl reference``: the oracle timed on the host cores, bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    probe = min(wl.E, 128)
+    t_probe, _, _ = oracle_run(wl, 0, probe)
+    budget = 90.0 / max(1, args.steps + args.warmup)            # whole run ~1.5 minutes
+    ns = int(min(wl.E, max(32, probe / max(t_probe, 1e-6) * min(budget, 10.0))))
+    from paper_2604_19906_b200 import inputs
+    host = inputs.host_case(wl, 0, ns)
+
+    def step():
+        if wl.op == "inv_helmholtz":
+            oracle.inv_helmholtz(host["S"], host["D"], host["u"])
+        else:
+            oracle.tpo_apply(host["A"], host["B"], host["C"], host["u"])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    cores = oracle.threads_used(0)
+    value = ns * args.steps / dt
+    sample = f"first {ns} of {wl.E} elements of {wl.name} per step on {cores} threads"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "elements_per_step": ns},
+            "gflops": value * wl.flops_per_element / 1e9,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ GPU arm
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3)
+    ap.add_argument("--elements", type=int, default=0, help="override E (profiling on small cases)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2604_19906_b200 import inputs
+    wl = inputs.CONFIGS[args.workload]
+    if args.elements:
+        wl = inputs.Workload(wl.index, wl.op, wl.n, wl.m, args.elements, wl.dtype)
+
+    if args.impl == "reference":
+        reference_arm(args, wl, rank)
+        return
+
+    # The oracle leg runs first, before any CUDA call (its OpenMP pool and the CUDA
+    # context do not interact, and the GPUs are not held while the host works).
+    base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        base, v_oracle, ns_oracle = cpu_baseline(wl)
+
+    import torch
+    from paper_2604_19906_b200 import build, ops, sharding
+    build.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    else:
+        dist = None
+    if world != args.gpus and rank == 0:
+        print(f"# note: --gpus {args.gpus} but WORLD_SIZE={world}", file=sys.stderr)
+
+    lib = ops.library()
+    e0, e1 = sharding.weak_range(wl.E, rank, world)
+    case = inputs.device_case(wl, dev, e0, e1)
+    E = wl.E
+    if wl.op == "inv_helmholtz":
+        v = torch.empty_like(case["u"])
+        a = (case["S"].data_ptr(), case["D"].data_ptr(), case["u"].data_ptr(), v.data_ptr(),
+             wl.n[0], E)
+        fn = lib.ekl_tpo_inv_helmholtz
+    else:
+        v = torch.empty((E,) + tuple(wl.m), dtype=torch.float64, device=dev)
+        a = (case["A"].data_ptr(), case["B"].data_ptr(), case["C"].data_ptr(),
+             case["u"].data_ptr(), v.data_ptr(), *wl.n, *wl.m, E)
+        fn = lib.ekl_tpo_apply
+    stream = torch.cuda.Stream(dev)
+    sp = stream.cuda_stream
+
+    def step():
+        st = fn(*a, sp)
+        if st:
+            raise ops.EklTpoError(st, "bench step")
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
+        torch.cuda.synchronize(dev)
+        props = torch.cuda.get_device_properties(dev)
+        sampler = ClockSampler(str(getattr(props, "uuid", "")), local_rank)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        per = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+        barrier()
+        torch.cuda.synchronize(dev)
+        sampler.start()
+        ev0.record(stream)
+        for k in range(args.steps):
+            per[k][0].record(stream)
+            step()
+            per[k][1].record(stream)
+        ev1.record(stream)
+        torch.cuda.synchronize(dev)
+        barrier()
+        clocks = sampler.stop()
+    total_ms = ev0.elapsed_time(ev1)
+    launch_ms = [p[0].elapsed_time(p[1]) for p in per]
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * E / (ms_per_step * 1e-3)
+
+    # ---------------------------------------------------------------- parity on the oracle's sample
+    max_rel_err = None
+    if base is not None:
+        import oracle
+        got = v[:ns_oracle].cpu().numpy()
+        max_rel_err = float(oracle.rel_err_per_element(got, v_oracle).max())
+
+    # ---------------------------------------------------------------- FP64 rate of this device, live
+    fp64_meas = None
+    if rank == 0:
+        import ctypes
+        sink = torch.empty(SM_COUNT * 8 * 256, dtype=torch.float64, device=dev)
+        flops = ctypes.c_double(0.0)
+        with torch.cuda.stream(stream):
+            best = None
+            for it in range(4):
+                s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s.record(stream)
+                lib.ekl_tpo_probe_fp64_fma.argtypes = None
+                rc = lib.ekl_tpo_probe_fp64_fma(ctypes.c_void_p(sink.data_ptr()), SM_COUNT * 8,
+                                                20000, ctypes.byref(flops), ctypes.c_void_p(sp))
+                e.record(stream)
+                torch.cuda.synchronize(dev)
+                if rc == 0 and it > 0:
+                    ms = s.elapsed_time(e)
+                    best = ms if best is None else min(best, ms)
+        if best:
+            fp64_meas = flops.value / (best * 1e-3) / 1e12
+
+    # ---------------------------------------------------------------- end to end with host buffers
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(torch, ops, wl, case, dev, stream, args.e2e_steps, world, dist)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = measured_peaks()
+    avg_launch_ms = statistics.fmean(launch_ms)
+    flops_launch = E * wl.flops_per_element
+    bytes_launch = E * wl.bytes_per_element
+    tf = flops_launch / (avg_launch_ms * 1e-3) / 1e12
+    gbs = bytes_launch / (avg_launch_ms * 1e-3) / 1e9
+    hbm_peak = float(peaks.get("hbm_gbs", HBM_FALLBACK_GBS))
+    t_alu = flops_launch / (FP64_PEAK_TFLOPS * 1e12)
+    t_hbm = bytes_launch / (hbm_peak * 1e9)
+    if t_alu >= t_hbm:
+        roof = {"bound": "alu", "achieved": tf, "peak": FP64_PEAK_TFLOPS, "unit": "TFLOP/s",
+                "frac": tf / FP64_PEAK_TFLOPS}
+    else:
+        roof = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
+                "frac": gbs / hbm_peak}
+    roof.update({
+        "traffic": None,
+        "kernel_ms": avg_launch_ms,
+        "peak_source": ("alu: 148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz; hbm: "
+                        f"MEASURED_PEAKS.json ({peak_src})"),
+        "fp64_tflops": tf, "fp64_peak_derived": FP64_PEAK_TFLOPS,
+        "fp64_peak_probe_tflops": fp64_meas,
+        "hbm_gbs": gbs, "hbm_peak_gbs": hbm_peak, "hbm_frac": gbs / hbm_peak,
+        "min_roof_ms": max(t_alu, t_hbm) * 1e3,
+        "frac_of_min_roof": max(t_alu, t_hbm) * 1e3 / avg_launch_ms})
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "elements_per_gpu": E,
+                       "l2": f"inputs larger than L2 ({bytes_launch / 1e9:.2f} GB per step)"
+                       if bytes_launch > 2 * 126e6 else "working set fits in L2 (warm)",
+                       "parallelism": f"elements sharded over {world} GPU(s), no collective"},
+            "gflops": value * wl.flops_per_element / 1e9,
+            "roofline": roof, "clocks": clocks, "gpu_launches": args.steps,
+            "max_rel_err_vs_oracle": max_rel_err}
+    if base is not None:
+        line["cpu_baseline"] = base
+    if e2e is not None:
+        line["e2e"] = e2e
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, ops, wl, case, dev, stream, steps, world, dist):
+    """Same metric through the public API with HOST buffers: every step copies u and D
+    from pinned host memory, runs the operator, and copies v back."""
+    E = wl.E
+    names = ("D", "u") if wl.op == "inv_helmholtz" else ("u",)
+    host_in = {k: torch.empty(case[k].shape, dtype=case[k].dtype, pin_memory=True).copy_(case[k])
+               for k in names}
+    out_shape = (E,) + tuple(wl.m)
+    host_out = torch.empty(out_shape, dtype=torch.float64, pin_memory=True)
+    mats = {k: case[k].cpu() for k in (("S",) if wl.op == "inv_helmholtz" else ("A", "B", "C"))}
+    torch.cuda.synchronize(dev)
+
+    def step():
+        if wl.op == "inv_helmholtz":
+            ops.ekl_tpo_inv_helmholtz_host(mats["S"], host_in["D"], host_in["u"], host_out,
+                                           device=dev)
+        else:
+            ops.ekl_tpo_apply_host(mats["A"], mats["B"], mats["C"], host_in["u"], host_out,
+                                   device=dev)
+
+    with torch.cuda.stream(stream):
+        step()
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            step()
+        torch.cuda.synchronize(dev)
+        dt = time.perf_counter() - t0
+    if dist is not None:
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values()) + \
+        sum(t.numel() * t.element_size() for t in mats.values())
+    d2h = host_out.numel() * host_out.element_size()
+    return {"value": world * E * steps / dt, "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": dt / steps * 1e3, "steps": steps,
+            "api": "ekl_tpo_*_host (pinned host buffers in, pinned host buffer out)"}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+/*
+ * ekl_tpo -- batched, sum-factorised spectral-element tensor-product operators
+ * for NVIDIA B200 (sm_100a).  C ABI; every pointer is a DEVICE pointer unless the
+ * name of the function ends in "_host".
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Arrays are dense, row-major (C order), last index fastest; the element
+ *    index e is the slowest one.  This is the row-major C ABI the paper's
+ *    kernels are linked through (Section 3, the remark on the column-major /
+ *    row-major difference next to the convective-flux listing).
+ *  - Kronecker ordering as in Eq. 1 of the paper: in (A (x) B (x) C) the last
+ *    factor acts on the fastest (contiguous) in-element axis,
+ *        ((A (x) B (x) C) x)[i,j,k] = sum_{l,m,n} A[i,l] B[j,m] C[k,n] x[l,m,n],
+ *    with every matrix stored [out, in] row-major.
+ *  - The result is the one the lifted ("reduction lifting", Section 5.2) sums
+ *    define mathematically; floating-point association inside the library is
+ *    unspecified (FMA is used), so results agree with a reference to rounding,
+ *    not bit for bit.
+ *  - Ownership: the caller owns every buffer.  Unless stated otherwise the
+ *    library allocates nothing, frees nothing and never synchronises: a call
+ *    validates its arguments on the host, enqueues work on `stream` and returns.
+ *    Buffers must stay valid until the stream has passed that work.  Inputs are
+ *    only read; the output is fully overwritten.
+ *  - Errors: a status code is returned; nothing is thrown, aborted or trapped,
+ *    and arguments that are accepted can never index out of bounds.  Validation
+ *    happens before anything is enqueued:
+ *        E > 0 and a null pointer                      -> EKL_TPO_ERR_NULL
+ *        an extent < 1, or E < 0                       -> EKL_TPO_ERR_SHAPE
+ *        extents too large for on-chip memory          -> EKL_TPO_ERR_UNSUPPORTED
+ *        pointer not aligned to its element type       -> EKL_TPO_ERR_ALIGN
+ *        output overlapping an input (see below)       -> EKL_TPO_ERR_OVERLAP
+ *        a CUDA runtime call failed                    -> EKL_TPO_ERR_CUDA
+ *    E == 0 is a successful no-op.  There is no CPU fallback of any kind.
+ */
+#ifndef EKL_TPO_H
+#define EKL_TPO_H
+
+#include <cuda_runtime_api.h>
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EKL_TPO_OK = 0,
+    EKL_TPO_ERR_NULL = 1,
+    EKL_TPO_ERR_SHAPE = 2,
+    EKL_TPO_ERR_UNSUPPORTED = 3,
+    EKL_TPO_ERR_ALIGN = 4,
+    EKL_TPO_ERR_OVERLAP = 5,
+    EKL_TPO_ERR_CUDA = 6
+} ekl_tpo_status;
+
+/*
+ * Inverse Helmholtz operator (the `inv_helm` kernel of Section 2.2 / Table 2; its
+ * forward stage is the lifted triple sum printed in Section 5.2):
+ *
+ *     v[e] = (S (x) S (x) S) . ( D[e] o ( (S^T (x) S^T (x) S^T) . u[e] ) ),   e = 0..E-1
+ *
+ *   S      [n,n]       one matrix shared by all elements and directions
+ *   D,u,v  [E,n,n,n]   D is multiplied pointwise (it holds the reciprocals)
+ *
+ * fp64.  `v == u` exactly (in place) is allowed; any other overlap of v with an
+ * input is rejected.  1 <= n; n is limited by shared memory (n <= 24 for fp64).
+ */
+ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const double* u,
+                                     double* v, int n, long long E, cudaStream_t stream);
+
+/*
+ * Forward rectangular tensor-product operator (the operator family of Eq. 1):
+ *
+ *     v[e] = (A (x) B (x) C) . u[e],   e = 0..E-1
+ *
+ *   A [m0,n0]  B [m1,n1]  C [m2,n2]     u [E,n0,n1,n2]     v [E,m0,m1,m2]
+ *
+ * fp64.  v must not overlap any input.
+ */
+ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
+                             const double* u, double* v,
+                             int n0, int n1, int n2, int m0, int m1, int m2,
+                             long long E, cudaStream_t stream);
+
+/* Single-precision twins of the two operators above (same layout and rules). */
+ekl_tpo_status ekl_tpo_inv_helmholtz_f32(const float* S, const float* D, const float* u,
+                                         float* v, int n, long long E, cudaStream_t stream);
+ekl_tpo_status ekl_tpo_apply_f32(const float* A, const float* B, const float* C,
+                                 const float* u, float* v,
+                                 int n0, int n1, int n2, int m0, int m1, int m2,
+                                 long long E, cudaStream_t stream);
+
+/*
+ * Host-buffer variants.  S (resp. A, B, C), D, u and v are HOST pointers; pinned
+ * (page-locked) memory is needed for the copies to overlap with the kernels, pageable
+ * memory works but serialises.  The E elements are cut into chunks; each chunk is
+ * copied into `workspace`, processed by the same kernels as the device-pointer entry
+ * point (Section 5.2 / Eq. 1 operators as above), and copied back, three chunks in
+ * flight (copy-in, compute, copy-out).
+ *
+ *   workspace        DEVICE scratch owned by the caller, 256-byte aligned, of
+ *   workspace_bytes  bytes.  Any size that holds the matrices plus three one-element
+ *                    slots is accepted (smaller -> EKL_TPO_ERR_UNSUPPORTED); larger
+ *                    workspaces give larger chunks.  ekl_tpo_host_workspace_bytes()
+ *                    returns the size for a wanted chunk length.  Its contents are
+ *                    scratch: undefined after the call, nothing to clear before it.
+ *
+ * The call enqueues everything and returns without synchronising when the host
+ * buffers are pinned; `stream` completes only after the last chunk of v has landed in
+ * host memory.  Two helper streams and a few events per device are created on first
+ * use (no device memory is allocated).  v == u (in place) is allowed for the inverse
+ * Helmholtz variant.  Calls are serialised by an internal lock while they enqueue; two
+ * calls sharing one workspace must be ordered on the same stream.
+ */
+ekl_tpo_status ekl_tpo_inv_helmholtz_host(const double* S, const double* D, const double* u,
+                                          double* v, int n, long long E, void* workspace,
+                                          size_t workspace_bytes, cudaStream_t stream);
+ekl_tpo_status ekl_tpo_apply_host(const double* A, const double* B, const double* C,
+                                  const double* u, double* v,
+                                  int n0, int n1, int n2, int m0, int m1, int m2,
+                                  long long E, void* workspace, size_t workspace_bytes,
+                                  cudaStream_t stream);
+
+/*
+ * Bytes of device workspace that let the host-buffer variants run with chunks of
+ * `chunk` elements: `n_inputs` per-element input fields of `in_elems_per_element`
+ * values each (2 for inverse Helmholtz: D and u; 1 for the forward operator), one output
+ * field of `out_elems_per_element` values, `matrix_elems` matrix entries in total,
+ * `elem_size` bytes per value.  Returns 0 for nonsensical arguments.
+ */
+size_t ekl_tpo_host_workspace_bytes(long long in_elems_per_element, int n_inputs,
+                                    long long out_elems_per_element, long long matrix_elems,
+                                    long long chunk, int elem_size);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* ekl_tpo_status_string(ekl_tpo_status status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int ekl_tpo_version(void);
+
+/* cudaError_t of the most recent EKL_TPO_ERR_CUDA returned on the calling thread. */
+int ekl_tpo_last_cuda_error(void);
+
+/*
+ * Measurement helper (no counterpart in the paper): enqueues `blocks` CTAs of 256
+ * threads, each thread running 16 independent chains of `iters` dependent fp64 FMAs
+ * in registers, and stores in *flops (HOST pointer, written before returning) the
+ * number of floating-point operations that launch performs.  `sink` is a device
+ * buffer of at least blocks*256 doubles that receives one value per thread.  Timing
+ * the launch gives the sustained FP64 FMA rate the roofline fractions refer to.
+ */
+ekl_tpo_status ekl_tpo_probe_fp64_fma(double* sink, int blocks, int iters, double* flops,
+                                      cudaStream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EKL_TPO_H */

@@ -1,0 +1,59 @@
+// Host-side kernel selection shared by the entry points.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstddef>
+
+namespace ekl {
+
+// Largest dynamic shared memory a CTA may opt into on sm_100.
+constexpr size_t kMaxSmemBytes = 227 * 1024;
+
+// Shared memory the run-time-sized inverse-Helmholtz kernel needs: S + two element buffers.
+inline size_t generic_ih_smem(int n, size_t elem) {
+    return ((size_t)n * n + 2 * (size_t)n * n * n) * elem;
+}
+
+// Largest cubic extent the library accepts for elements of `elem` bytes.
+inline int max_cubic_extent(size_t elem) {
+    int n = 1;
+    while (generic_ih_smem(n + 1, elem) <= kMaxSmemBytes) ++n;
+    return n;
+}
+
+// Elements of one ping-pong buffer of the run-time-sized forward kernel.
+inline size_t generic_apply_buf(int n0, int n1, int n2, int m1, int m2) {
+    size_t a = (size_t)n0 * n1 * n2, b = (size_t)n0 * n1 * m2, c = (size_t)n0 * m1 * m2;
+    size_t even = a > c ? a : c;  // buffer 0 holds u then q, buffer 1 holds p
+    return even > b ? even : b;
+}
+
+inline size_t generic_apply_smem(int n0, int n1, int n2, int m0, int m1, int m2, size_t elem) {
+    return ((size_t)m0 * n0 + (size_t)m1 * n1 + (size_t)m2 * n2 +
+            2 * generic_apply_buf(n0, n1, n2, m1, m2)) * elem;
+}
+
+inline bool apply_fits(int n0, int n1, int n2, int m0, int m1, int m2, size_t elem) {
+    // guard the products against overflow before comparing
+    const double est = ((double)n0 * n1 * n2 + (double)n0 * n1 * m2 + (double)n0 * m1 * m2 +
+                        (double)m0 * n0 + (double)m1 * n1 + (double)m2 * n2) * (double)elem;
+    if (est > 4.0 * (double)kMaxSmemBytes) return false;
+    if ((double)m0 * m1 * m2 > 2.0e9) return false;
+    return generic_apply_smem(n0, n1, n2, m0, m1, m2, elem) <= kMaxSmemBytes;
+}
+
+// Records the cudaError_t that ekl_tpo_last_cuda_error() reports for the calling thread.
+void set_last_cuda_error(int err);
+
+// Number of SMs of the current device (cached per device).
+int sm_count();
+
+template <typename T>
+cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
+                                 cudaStream_t stream);
+
+template <typename T>
+cudaError_t launch_apply(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
+                         int n2, int m0, int m1, int m2, long long E, cudaStream_t stream);
+
+}  // namespace ekl

@@ -1,0 +1,228 @@
+"""Thin Python binding of the C-ABI library (``include/ekl_tpo.h``).
+
+Argument marshalling only: every function here takes CUDA tensors, checks dtype /
+device / contiguity, and passes raw device pointers, extents and the current CUDA
+stream to the entry point of the same name in ``lib/libekl_tpo.so``.  All arithmetic
+runs in the library's kernels; there is no fallback -- if the library is missing or a
+call is rejected, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_LIBPATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libekl_tpo.so")
+_lib = None
+
+STATUS_NAMES = {0: "EKL_TPO_OK", 1: "EKL_TPO_ERR_NULL", 2: "EKL_TPO_ERR_SHAPE",
+                3: "EKL_TPO_ERR_UNSUPPORTED", 4: "EKL_TPO_ERR_ALIGN", 5: "EKL_TPO_ERR_OVERLAP",
+                6: "EKL_TPO_ERR_CUDA"}
+
+
+class EklTpoError(RuntimeError):
+    """A library call returned a status other than EKL_TPO_OK."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib = library()
+        msg = lib.ekl_tpo_status_string(status).decode()
+        extra = f", cudaError {lib.ekl_tpo_last_cuda_error()}" if status == 6 else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg}{extra})")
+
+
+def library() -> ctypes.CDLL:
+    """The loaded C-ABI library with argument types declared (raises if it is not built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIBPATH):
+            raise RuntimeError(
+                f"{_LIBPATH} is missing: build it with `python -m paper_2604_19906_b200.build` "
+                "(there is no fallback implementation)")
+        lib = ctypes.CDLL(_LIBPATH)
+        vp, i, ll = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong
+        for name in ("ekl_tpo_inv_helmholtz", "ekl_tpo_inv_helmholtz_f32"):
+            f = getattr(lib, name)
+            f.argtypes = [vp, vp, vp, vp, i, ll, vp]
+            f.restype = i
+        for name in ("ekl_tpo_apply", "ekl_tpo_apply_f32"):
+            f = getattr(lib, name)
+            f.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, ll, vp]
+            f.restype = i
+        lib.ekl_tpo_status_string.argtypes = [i]
+        lib.ekl_tpo_status_string.restype = ctypes.c_char_p
+        lib.ekl_tpo_version.restype = i
+        lib.ekl_tpo_last_cuda_error.restype = i
+        _lib = lib
+    return _lib
+
+
+def _dev_ptr(t: torch.Tensor, name: str, dtype: torch.dtype, device: torch.device) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if t.device != device:
+        raise ValueError(f"{name} is on {t.device}, expected {device}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous (row-major)")
+    return t.data_ptr()
+
+
+def _stream(device: torch.device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _inv_helmholtz(fn_name, dtype, S, D, u, out):
+    if u.dim() != 4 or S.dim() != 2:
+        raise ValueError("S must be [n,n] and u [E,n,n,n]")
+    E, n = u.shape[0], S.shape[0]
+    if tuple(S.shape) != (n, n) or tuple(u.shape[1:]) != (n, n, n) or D.shape != u.shape:
+        raise ValueError("expected S [n,n] and D,u [E,n,n,n]")
+    dev = u.device
+    if out is None:
+        out = torch.empty_like(u)
+    elif out.shape != u.shape:
+        raise ValueError("out must have the shape of u")
+    ptrs = [_dev_ptr(t, nm, dtype, dev) for t, nm in ((S, "S"), (D, "D"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = getattr(library(), fn_name)(*ptrs, n, E, _stream(dev))
+    if st:
+        raise EklTpoError(st, fn_name)
+    return out
+
+
+def ekl_tpo_inv_helmholtz(S, D, u, out=None):
+    """``v[e] = (S⊗S⊗S)·(D[e] ∘ ((Sᵀ⊗Sᵀ⊗Sᵀ)·u[e]))`` in fp64 on the current stream.
+    ``out`` may be ``u`` itself (in place)."""
+    return _inv_helmholtz("ekl_tpo_inv_helmholtz", torch.float64, S, D, u, out)
+
+
+def ekl_tpo_inv_helmholtz_f32(S, D, u, out=None):
+    """Single-precision twin of :func:`ekl_tpo_inv_helmholtz`."""
+    return _inv_helmholtz("ekl_tpo_inv_helmholtz_f32", torch.float32, S, D, u, out)
+
+
+def _apply(fn_name, dtype, A, B, C, u, out):
+    if u.dim() != 4 or A.dim() != 2 or B.dim() != 2 or C.dim() != 2:
+        raise ValueError("A,B,C must be matrices and u [E,n0,n1,n2]")
+    (m0, n0), (m1, n1), (m2, n2) = A.shape, B.shape, C.shape
+    E = u.shape[0]
+    if tuple(u.shape[1:]) != (n0, n1, n2):
+        raise ValueError("u must be [E,n0,n1,n2] with n_d the column counts of A,B,C")
+    dev = u.device
+    if out is None:
+        out = torch.empty((E, m0, m1, m2), dtype=dtype, device=dev)
+    elif tuple(out.shape) != (E, m0, m1, m2):
+        raise ValueError("out must be [E,m0,m1,m2]")
+    ptrs = [_dev_ptr(t, nm, dtype, dev)
+            for t, nm in ((A, "A"), (B, "B"), (C, "C"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = getattr(library(), fn_name)(*ptrs, n0, n1, n2, m0, m1, m2, E, _stream(dev))
+    if st:
+        raise EklTpoError(st, fn_name)
+    return out
+
+
+def ekl_tpo_apply(A, B, C, u, out=None):
+    """``v[e] = (A⊗B⊗C)·u[e]`` in fp64 on the current stream."""
+    return _apply("ekl_tpo_apply", torch.float64, A, B, C, u, out)
+
+
+def ekl_tpo_apply_f32(A, B, C, u, out=None):
+    """Single-precision twin of :func:`ekl_tpo_apply`."""
+    return _apply("ekl_tpo_apply_f32", torch.float32, A, B, C, u, out)
+
+
+def ekl_tpo_version() -> int:
+    return int(library().ekl_tpo_version())
+
+
+# ----------------------------------------------------------------------------- host buffers
+
+_workspaces: dict = {}
+
+
+def _declare_host(lib):
+    if getattr(lib, "_host_declared", False):
+        return
+    vp, i, ll, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_size_t
+    lib.ekl_tpo_inv_helmholtz_host.argtypes = [vp, vp, vp, vp, i, ll, vp, sz, vp]
+    lib.ekl_tpo_inv_helmholtz_host.restype = i
+    lib.ekl_tpo_apply_host.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, ll, vp, sz, vp]
+    lib.ekl_tpo_apply_host.restype = i
+    lib.ekl_tpo_host_workspace_bytes.argtypes = [ll, i, ll, ll, ll, i]
+    lib.ekl_tpo_host_workspace_bytes.restype = sz
+    lib._host_declared = True
+
+
+def host_workspace(device, nbytes: int) -> torch.Tensor:
+    """A cached device scratch buffer of at least ``nbytes`` bytes on ``device`` (device
+    memory comes from torch; the library itself allocates none)."""
+    dev = torch.device(device)
+    key = (dev.type, dev.index)
+    ws = _workspaces.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        _workspaces[key] = ws
+    return ws
+
+
+def _host_ptr(t: torch.Tensor, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError(f"{name} must be a CPU tensor")
+    if t.dtype != torch.float64:
+        raise TypeError(f"{name} must be float64")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous (row-major)")
+    return t.data_ptr()
+
+
+def ekl_tpo_inv_helmholtz_host(S, D, u, out, device="cuda:0", chunk: int = 2048,
+                               workspace: torch.Tensor | None = None):
+    """Inverse Helmholtz with HOST tensors in and out (pinned memory lets copies and
+    kernels overlap).  Enqueues on the current stream of ``device`` and returns; the
+    result is complete once that stream has been synchronised."""
+    lib = library()
+    _declare_host(lib)
+    E, n = u.shape[0], S.shape[0]
+    if tuple(S.shape) != (n, n) or tuple(u.shape[1:]) != (n, n, n) or D.shape != u.shape \
+            or out.shape != u.shape:
+        raise ValueError("expected S [n,n] and D,u,out [E,n,n,n]")
+    dev = torch.device(device)
+    if workspace is None:
+        need = lib.ekl_tpo_host_workspace_bytes(n ** 3, 2, n ** 3, n * n, max(1, min(chunk, E)), 8)
+        workspace = host_workspace(dev, need)
+    ptrs = [_host_ptr(t, nm) for t, nm in ((S, "S"), (D, "D"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = lib.ekl_tpo_inv_helmholtz_host(*ptrs, n, E, workspace.data_ptr(), workspace.numel(),
+                                            _stream(dev))
+    if st:
+        raise EklTpoError(st, "ekl_tpo_inv_helmholtz_host")
+    return out
+
+
+def ekl_tpo_apply_host(A, B, C, u, out, device="cuda:0", chunk: int = 4096,
+                       workspace: torch.Tensor | None = None):
+    """Forward operator with HOST tensors in and out; see
+    :func:`ekl_tpo_inv_helmholtz_host`."""
+    lib = library()
+    _declare_host(lib)
+    (m0, n0), (m1, n1), (m2, n2) = A.shape, B.shape, C.shape
+    E = u.shape[0]
+    if tuple(u.shape[1:]) != (n0, n1, n2) or tuple(out.shape) != (E, m0, m1, m2):
+        raise ValueError("expected u [E,n0,n1,n2] and out [E,m0,m1,m2]")
+    dev = torch.device(device)
+    if workspace is None:
+        need = lib.ekl_tpo_host_workspace_bytes(n0 * n1 * n2, 1, m0 * m1 * m2,
+                                                m0 * n0 + m1 * n1 + m2 * n2,
+                                                max(1, min(chunk, E)), 8)
+        workspace = host_workspace(dev, need)
+    ptrs = [_host_ptr(t, nm) for t, nm in ((A, "A"), (B, "B"), (C, "C"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = lib.ekl_tpo_apply_host(*ptrs, n0, n1, n2, m0, m1, m2, E, workspace.data_ptr(),
+                                    workspace.numel(), _stream(dev))
+    if st:
+        raise EklTpoError(st, "ekl_tpo_apply_host")
+    return out

@@ -1,0 +1,110 @@
+"""The C-ABI library loads, exports what include/*.h declares, and rejects bad
+arguments on the host before anything touches a device (no GPU needed: every call
+below returns from validation)."""
+import ctypes
+import glob
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_19906_b200 import build, ops
+    build.build()
+    return ops.library()
+
+
+def declared_symbols():
+    names = set()
+    for h in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = re.sub(r"/\*.*?\*/", "", open(h).read(), flags=re.S)
+        names |= set(re.findall(r"\b(ekl_tpo_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert {"ekl_tpo_inv_helmholtz", "ekl_tpo_apply", "ekl_tpo_inv_helmholtz_f32",
+            "ekl_tpo_apply_f32", "ekl_tpo_status_string", "ekl_tpo_version",
+            "ekl_tpo_last_cuda_error"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/ but not exported"
+
+
+def test_version_and_status_strings(lib):
+    assert lib.ekl_tpo_version() >= 100
+    seen = {lib.ekl_tpo_status_string(s) for s in range(7)}
+    assert len(seen) == 7 and all(seen)
+    assert lib.ekl_tpo_status_string(99)
+
+
+P = 0x7F0000001000          # a made-up, suitably aligned "device" address: never dereferenced
+
+
+@pytest.mark.parametrize("fn,w", [("ekl_tpo_inv_helmholtz", 8), ("ekl_tpo_inv_helmholtz_f32", 4)])
+def test_inv_helmholtz_validation(lib, fn, w):
+    f = getattr(lib, fn)
+    OK, NULL, SHAPE, UNSUP, ALIGN, OVERLAP = 0, 1, 2, 3, 4, 5
+    n, E = 4, 10
+    field = E * n ** 3 * w
+    S, D, u, v = P, P + 0x1000, P + 0x1000 + field, P + 0x1000 + 2 * field
+    assert f(S, D, u, v, 0, E, None) == SHAPE
+    assert f(S, D, u, v, -3, E, None) == SHAPE
+    assert f(S, D, u, v, n, -1, None) == SHAPE
+    assert f(None, None, None, None, n, 0, None) == OK          # E == 0 is a no-op
+    assert f(None, D, u, v, n, E, None) == NULL
+    assert f(S, D, u, None, n, E, None) == NULL
+    assert f(S, D, u, v, 1000, E, None) == UNSUP
+    assert f(S, D, u, v, 25 if w == 8 else 31, E, None) == UNSUP
+    assert f(S, D, u + w // 2, v, n, E, None) == ALIGN
+    assert f(S, D, u, v + 1, n, E, None) == ALIGN
+    assert f(S, D, u, D, n, E, None) == OVERLAP                  # v aliases D
+    assert f(S, D, u, u + w, n, E, None) == OVERLAP              # v partially overlaps u
+    assert f(S, D, u, S, n, E, None) == OVERLAP
+    assert f(S, D, u, D + field - w, n, E, None) == OVERLAP      # tail of D
+
+
+@pytest.mark.parametrize("fn,w", [("ekl_tpo_apply", 8), ("ekl_tpo_apply_f32", 4)])
+def test_apply_validation(lib, fn, w):
+    f = getattr(lib, fn)
+    OK, NULL, SHAPE, UNSUP, ALIGN, OVERLAP = 0, 1, 2, 3, 4, 5
+    E = 6
+    A, B, C = P, P + 0x400, P + 0x800
+    u = P + 0x1000
+    v = u + E * 8 ** 3 * w
+    dims = (8, 8, 8, 12, 12, 12)
+    assert f(A, B, C, u, v, 8, 8, 0, 12, 12, 12, E, None) == SHAPE
+    assert f(A, B, C, u, v, 8, 8, 8, 12, -1, 12, E, None) == SHAPE
+    assert f(A, B, C, u, v, *dims, -2, None) == SHAPE
+    assert f(None, None, None, None, None, *dims, 0, None) == OK
+    assert f(A, None, C, u, v, *dims, E, None) == NULL
+    assert f(A, B, C, u, v, 64, 64, 64, 64, 64, 64, E, None) == UNSUP
+    assert f(A, B, C, u, v, 40000, 40000, 40000, 40000, 40000, 40000, E, None) == UNSUP
+    assert f(A, B, C + 2, u, v, *dims, E, None) == ALIGN
+    assert f(A, B, C, u, u, *dims, E, None) == OVERLAP           # no in-place for apply
+    assert f(A, B, C, u, v - w, *dims, E, None) == OVERLAP
+    assert f(A, B, C, u, A, *dims, E, None) == OVERLAP
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    from paper_2604_19906_b200 import ops
+    monkeypatch.setattr(ops, "_lib", None)
+    monkeypatch.setattr(ops, "_LIBPATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        ops.library()
+
+
+def test_product_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2604_19906_b200")
+    for path in glob.glob(os.path.join(pkg, "**", "*"), recursive=True):
+        if path.endswith((".py", ".cu", ".cuh", ".h")):
+            text = open(path).read()
+            assert "import oracle" not in text and "from oracle" not in text, path
+            assert "tpo_oracle" not in text, path
+    for path in glob.glob(os.path.join(ROOT, "oracle", "*")):
+        if path.endswith((".py", ".c", ".h")):
+            assert "paper_2604_19906_b200" not in open(path).read(), path

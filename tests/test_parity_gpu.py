@@ -1,0 +1,241 @@
+"""GPU parity: the CUDA library (through its C ABI, via the thin binding) against the
+CPU oracle on the same seeded inputs.
+
+Bar: max over elements of ‖v_e − v̂_e‖₂/‖v̂_e‖₂ ≤ 1e-12 in fp64 and ≤ 1e-5 in fp32,
+v̂ = oracle (for fp32 the oracle widens the fp32 inputs and computes in fp64).
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL64 = 1e-12
+TOL32 = 1e-5
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    import oracle
+    from paper_2604_19906_b200 import build, inputs, ops
+    build.build()
+    assert torch.cuda.is_available()
+    return {"torch": torch, "oracle": oracle, "inputs": inputs, "ops": ops,
+            "dev": torch.device("cuda:0")}
+
+
+def rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def to_dev(env, a, dtype=None):
+    t = env["torch"].from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.to(env["dev"])
+
+
+def synth_ih(n, E, seed):
+    g = rng(seed)
+    S, _ = np.linalg.qr(g.standard_normal((n, n)))
+    lam = g.uniform(0.1, 2.0, n)
+    c = g.uniform(0.5, 1.5, E)
+    D = 1.0 / (((lam[:, None, None] + lam[None, :, None]) + lam[None, None, :])[None]
+               + c[:, None, None, None])
+    u = g.uniform(-1, 1, (E, n, n, n))
+    return np.ascontiguousarray(S), D, u
+
+
+# --------------------------------------------------------------------------- inverse Helmholtz
+
+@pytest.mark.parametrize("n", list(range(1, 17)) + [20, 24])
+@pytest.mark.parametrize("E", [1, 2, 3, 5, 37, 301])
+def test_inv_helmholtz_f64_small(env, n, E):
+    if n >= 20 and E > 37:
+        pytest.skip("large n covered at small E")
+    S, D, u = synth_ih(n, E, 1000 * n + E)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    got = env["ops"].ekl_tpo_inv_helmholtz(to_dev(env, S), to_dev(env, D), to_dev(env, u))
+    env["torch"].cuda.synchronize()
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy(), want)
+    assert err.max() <= TOL64, (n, E, err.max())
+
+
+@pytest.mark.parametrize("n", [2, 4, 7, 8, 12, 14, 16])
+def test_inv_helmholtz_nonorthogonal_S_pins_transposes(env, n):
+    """A non-orthogonal, non-symmetric S separates S from Sᵀ in both stages."""
+    g = rng(50 + n)
+    E = 33
+    S = g.standard_normal((n, n)) / np.sqrt(n)
+    D = g.uniform(0.1, 1.3, (E, n, n, n))
+    u = g.uniform(-1, 1, (E, n, n, n))
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    got = env["ops"].ekl_tpo_inv_helmholtz(to_dev(env, S), to_dev(env, D), to_dev(env, u))
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy(), want)
+    assert err.max() <= TOL64
+
+
+@pytest.mark.parametrize("n", [3, 4, 8, 12, 14])
+def test_inv_helmholtz_f32(env, n):
+    torch = env["torch"]
+    E = 65
+    S, D, u = synth_ih(n, E, 77 + n)
+    S32, D32, u32 = (x.astype(np.float32) for x in (S, D, u))
+    want = env["oracle"].inv_helmholtz(S32, D32, u32)          # widened, computed in fp64
+    got = env["ops"].ekl_tpo_inv_helmholtz_f32(to_dev(env, S32), to_dev(env, D32), to_dev(env, u32))
+    assert got.dtype == torch.float32
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().astype(np.float64), want)
+    assert err.max() <= TOL32
+
+
+@pytest.mark.parametrize("n", [4, 8, 12, 14])
+def test_inv_helmholtz_exact_special_cases(env, n):
+    """S = I gives D∘u bit for bit (every extra term is ×0, +0); a permutation matrix
+    gives an exact permuted, scaled copy."""
+    g = rng(5 + n)
+    E = 19
+    D = g.uniform(0.1, 1.3, (E, n, n, n))
+    u = g.uniform(-1, 1, (E, n, n, n))
+    got = env["ops"].ekl_tpo_inv_helmholtz(to_dev(env, np.eye(n)), to_dev(env, D), to_dev(env, u))
+    assert np.array_equal(got.cpu().numpy(), D * u)
+    perm = g.permutation(n)
+    S = np.zeros((n, n))
+    S[np.arange(n), perm] = 1.0
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    got = env["ops"].ekl_tpo_inv_helmholtz(to_dev(env, S), to_dev(env, D), to_dev(env, u))
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("n,E", [(4, 64), (8, 777), (12, 150), (14, 149), (14, 300)])
+def test_inv_helmholtz_in_place_guards_and_repeatability(env, n, E):
+    """v == u in place; canaries around v untouched; NaN-prefilled output fully
+    overwritten; two runs bitwise identical (no races, no unwritten outputs)."""
+    torch = env["torch"]
+    S, D, u = synth_ih(n, E, 9 + n)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    Sd, Dd, ud = to_dev(env, S), to_dev(env, D), to_dev(env, u)
+    pad = 512
+    big = torch.full((E * n ** 3 + 2 * pad,), float("nan"), dtype=torch.float64, device=env["dev"])
+    big[:pad] = 12345.0
+    big[-pad:] = 54321.0
+    out = big[pad:-pad].view(E, n, n, n)
+    env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud, out=out)
+    first = out.clone()
+    out.fill_(float("nan"))
+    env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud, out=out)
+    assert torch.equal(first, out)
+    assert bool((big[:pad] == 12345.0).all()) and bool((big[-pad:] == 54321.0).all())
+    assert env["oracle"].rel_err_per_element(out.cpu().numpy(), want).max() <= TOL64
+    inplace = ud.clone()
+    env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, inplace, out=inplace)
+    assert torch.equal(inplace, first)
+
+
+def test_element_permutation_and_batch_independence(env):
+    torch = env["torch"]
+    n, E = 14, 130
+    S, D, u = synth_ih(n, E, 4242)
+    Sd, Dd, ud = to_dev(env, S), to_dev(env, D), to_dev(env, u)
+    full = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud)
+    p = torch.from_numpy(rng(1).permutation(E)).to(env["dev"])
+    shuf = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd[p].contiguous(), ud[p].contiguous())
+    assert torch.equal(shuf, full[p])
+
+
+# --------------------------------------------------------------------------- forward operator
+
+SHAPES = [((2, 3, 4), (5, 2, 3)), ((8, 8, 8), (12, 12, 12)), ((12, 12, 12), (8, 8, 8)),
+          ((1, 1, 1), (1, 1, 1)), ((7, 1, 5), (2, 9, 3)), ((4, 4, 4), (4, 4, 4)),
+          ((14, 14, 14), (14, 14, 14)), ((5, 6, 7), (7, 6, 5)), ((16, 3, 9), (3, 16, 2))]
+
+
+@pytest.mark.parametrize("nn,mm", SHAPES)
+@pytest.mark.parametrize("E", [1, 3, 130])
+def test_apply_f64(env, nn, mm, E):
+    g = rng(hash((nn, mm, E)) % 10000)
+    A, B, C = (g.standard_normal((mm[d], nn[d])) / np.sqrt(nn[d]) for d in range(3))
+    u = g.uniform(-1, 1, (E,) + nn)
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C, u)))
+    assert tuple(got.shape) == (E,) + mm
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+
+
+@pytest.mark.parametrize("nn,mm", SHAPES[:3])
+def test_apply_f32(env, nn, mm):
+    g = rng(3)
+    E = 50
+    A, B, C = ((g.standard_normal((mm[d], nn[d])) / np.sqrt(nn[d])).astype(np.float32)
+               for d in range(3))
+    u = g.uniform(-1, 1, (E,) + nn).astype(np.float32)
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    got = env["ops"].ekl_tpo_apply_f32(*(to_dev(env, x) for x in (A, B, C, u)))
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().astype(np.float64), want)
+    assert err.max() <= TOL32
+
+
+def test_apply_selection_matrices_gather_exactly(env):
+    g = rng(8)
+    nn, mm = (8, 8, 8), (12, 12, 12)
+    rows = [g.integers(0, nn[d], size=mm[d]) for d in range(3)]
+    A, B, C = (np.eye(nn[d])[rows[d]] for d in range(3))
+    u = g.uniform(-1, 1, (40,) + nn)
+    want = u[:, rows[0]][:, :, rows[1]][:, :, :, rows[2]]
+    got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C, u)))
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_apply_guards_and_repeatability(env):
+    torch = env["torch"]
+    g = rng(12)
+    nn, mm, E = (8, 8, 8), (12, 12, 12), 333
+    A, B, C = (g.standard_normal((mm[d], nn[d])) / np.sqrt(nn[d]) for d in range(3))
+    u = g.uniform(-1, 1, (E,) + nn)
+    dev = [to_dev(env, x) for x in (A, B, C, u)]
+    pad = 512
+    big = torch.full((E * 12 ** 3 + 2 * pad,), float("nan"), dtype=torch.float64, device=env["dev"])
+    big[:pad] = 1.5
+    big[-pad:] = 2.5
+    out = big[pad:-pad].view(E, 12, 12, 12)
+    env["ops"].ekl_tpo_apply(*dev, out=out)
+    first = out.clone()
+    out.fill_(float("nan"))
+    env["ops"].ekl_tpo_apply(*dev, out=out)
+    assert torch.equal(first, out)
+    assert bool((big[:pad] == 1.5).all()) and bool((big[-pad:] == 2.5).all())
+    assert not bool(torch.isnan(out).any())
+
+
+# --------------------------------------------------------------------------- binding / status paths
+
+def test_runtime_argument_errors_raise(env):
+    torch, ops = env["torch"], env["ops"]
+    n, E = 4, 8
+    S = torch.eye(n, dtype=torch.float64, device=env["dev"])
+    u = torch.zeros(E, n, n, n, dtype=torch.float64, device=env["dev"])
+    with pytest.raises(ops.EklTpoError, match="OVERLAP"):
+        ops.ekl_tpo_inv_helmholtz(S, u, u.clone(), out=u)        # D aliases v
+    with pytest.raises(TypeError):
+        ops.ekl_tpo_inv_helmholtz(S.float(), u, u)
+    with pytest.raises(TypeError):
+        ops.ekl_tpo_inv_helmholtz(S.cpu(), u, u)
+    with pytest.raises(ValueError):
+        ops.ekl_tpo_inv_helmholtz(S, u, u.transpose(1, 2))
+    big = torch.zeros(1, 26, 26, 26, dtype=torch.float64, device=env["dev"])
+    with pytest.raises(ops.EklTpoError, match="UNSUPPORTED"):
+        ops.ekl_tpo_inv_helmholtz(torch.eye(26, dtype=torch.float64, device=env["dev"]), big, big)
+    empty = torch.zeros(0, n, n, n, dtype=torch.float64, device=env["dev"])
+    assert ops.ekl_tpo_inv_helmholtz(S, empty, empty).shape == (0, n, n, n)
+
+
+def test_device_input_generators_match_the_host_bit_for_bit(env):
+    inputs = env["inputs"]
+    for idx in (0, 1, 4):
+        wl = inputs.CONFIGS[idx]
+        e0, e1 = 5, min(wl.E, 45)
+        host = inputs.host_case(wl, e0, e1)
+        dev = inputs.device_case(wl, env["dev"], e0, e1)
+        for key in host:
+            h = host[key]
+            d = dev[key].cpu().numpy() if hasattr(dev[key], "cpu") else dev[key]
+            assert np.array_equal(h, d), (idx, key)

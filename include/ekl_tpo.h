@@ -132,6 +132,42 @@ size_t ekl_tpo_host_workspace_bytes(long long in_elems_per_element, int n_inputs
                                     long long out_elems_per_element, long long matrix_elems,
                                     long long chunk, int elem_size);
 
+/*
+ * Inverse Helmholtz with HOST buffers and no device allocation anywhere (the paper has
+ * no counterpart: this entry point exists for deployment, not for the method).
+ *
+ * For callers that cannot obtain device memory when they need the operator -- a solver
+ * step running inside a memory budget fixed at start-up, a plug-in inside an
+ * application that owns the GPU heap, a latency-critical path where cudaMalloc (which
+ * may synchronise the device, or fail once memory is fragmented) is off limits -- and
+ * who therefore have no workspace to give ekl_tpo_inv_helmholtz_host.  Same operator,
+ * layout, argument meaning and status codes as ekl_tpo_inv_helmholtz_host; S, D, u, v
+ * are HOST pointers (pinned memory makes the copies asynchronous).  The staging area is
+ * a fixed array of EKL_TPO_STATIC_SCRATCH_BYTES bytes inside the library image; every
+ * GPU that loads the library holds that much memory until the process exits.  The call
+ * and everything it calls allocate and free nothing.
+ *
+ *  - Limit: the whole call is staged at once, so it needs
+ *        roundup256(8 n^2) + 3 * roundup256(8 E n^3)  <=  EKL_TPO_STATIC_SCRATCH_BYTES
+ *    (about 509 elements at n = 14, 2730 at n = 8).  Anything larger is rejected with
+ *    EKL_TPO_ERR_UNSUPPORTED before any work is enqueued; split such a batch into
+ *    several calls on one stream, or use ekl_tpo_inv_helmholtz_host.
+ *  - Set-up: the first call on each device looks up the staging area's device address
+ *    (with that device current) and keeps it.  Make that first call outside any stream
+ *    capture; `stream` must belong to the current device.
+ *  - Sharing: all calls on a device use the same staging area, and it keeps whatever
+ *    the previous call left there.  Nothing has to be cleared -- each call overwrites
+ *    all it reads -- but two calls that can run at the same time on the GPU (different
+ *    streams without an ordering between them) race on it and corrupt each other.
+ *    Issue them on one stream, or order them with events.
+ *  - Work is enqueued on `stream` only (copy in, kernel, copy out, in that order); the
+ *    result is in v once `stream` has reached the end of the call.  v == u is allowed.
+ */
+#define EKL_TPO_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+ekl_tpo_status ekl_tpo_inv_helmholtz_host_static(const double* S, const double* D,
+                                                 const double* u, double* v, int n,
+                                                 long long E, cudaStream_t stream);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 const char* ekl_tpo_status_string(ekl_tpo_status status);
 

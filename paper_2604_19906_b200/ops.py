@@ -226,3 +226,41 @@ def ekl_tpo_apply_host(A, B, C, u, out, device="cuda:0", chunk: int = 4096,
     if st:
         raise EklTpoError(st, "ekl_tpo_apply_host")
     return out
+
+
+# ----------------------------------------------------------------------------- no allocation
+
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+
+
+def static_scratch_need(n: int, E: int) -> int:
+    """Bytes of the library's fixed staging area a call with these sizes occupies."""
+    r = lambda x: (x + 255) // 256 * 256
+    return r(8 * n * n) + 3 * r(8 * E * n ** 3)
+
+
+def ekl_tpo_inv_helmholtz_host_static(S, D, u, out, device="cuda:0"):
+    """Inverse Helmholtz with HOST tensors in and out, for callers that cannot allocate
+    device memory: the call is staged in a fixed array inside the library, so neither
+    this wrapper nor the library allocates anything on the GPU.  The whole batch must
+    fit in that array (``static_scratch_need(n, E) <= STATIC_SCRATCH_BYTES``); larger
+    batches raise.  Calls share the array, so keep them on one stream."""
+    lib = library()
+    fn = lib.ekl_tpo_inv_helmholtz_host_static
+    fn.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p]
+    fn.restype = ctypes.c_int
+    E, n = u.shape[0], S.shape[0]
+    if tuple(S.shape) != (n, n) or tuple(u.shape[1:]) != (n, n, n) or D.shape != u.shape \
+            or out.shape != u.shape:
+        raise ValueError("expected S [n,n] and D,u,out [E,n,n,n]")
+    dev = torch.device(device)
+    ptrs = [_host_ptr(t, nm) for t, nm in ((S, "S"), (D, "D"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = fn(*ptrs, n, E, _stream(dev))
+    if st == 3 and static_scratch_need(n, E) > STATIC_SCRATCH_BYTES:
+        raise EklTpoError(st, "ekl_tpo_inv_helmholtz_host_static: the batch needs "
+                              f"{static_scratch_need(n, E)} bytes of staging, the fixed area "
+                              f"holds {STATIC_SCRATCH_BYTES}")
+    if st:
+        raise EklTpoError(st, "ekl_tpo_inv_helmholtz_host_static")
+    return out

@@ -48,6 +48,11 @@ void set_last_cuda_error(int err);
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
+// Tensor-path inverse Helmholtz (fp64).  Returns false if there is no instance for this n
+// or the pointers do not meet its alignment needs; otherwise launches and sets *err.
+bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
+                        long long E, cudaStream_t stream, cudaError_t* err);
+
 template <typename T>
 cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
                                  cudaStream_t stream);

@@ -1,4 +1,7 @@
 // Kernel selection and launch configuration.
+#include <cstdlib>
+#include <cstring>
+
 #include "dispatch.h"
 #include "generic_kernel.cuh"
 
@@ -67,10 +70,27 @@ cudaError_t launch_apply_generic(const T* A, const T* B, const T* C, const T* u,
 
 }  // namespace
 
-template <typename T>
-cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
-                                 cudaStream_t stream) {
-    return launch_ih_generic<T>(S, D, u, v, n, E, stream);
+// EKL_TPO_VARIANT=generic forces the run-time-sized kernels (A/B measurements).
+static bool tuned_allowed() {
+    static const bool allowed = [] {
+        const char* v = std::getenv("EKL_TPO_VARIANT");
+        return !(v && std::strcmp(v, "generic") == 0);
+    }();
+    return allowed;
+}
+
+template <>
+cudaError_t launch_inv_helmholtz<double>(const double* S, const double* D, const double* u,
+                                         double* v, int n, long long E, cudaStream_t stream) {
+    cudaError_t err = cudaSuccess;
+    if (tuned_allowed() && try_launch_ih_dmma(S, D, u, v, n, E, stream, &err)) return err;
+    return launch_ih_generic<double>(S, D, u, v, n, E, stream);
+}
+
+template <>
+cudaError_t launch_inv_helmholtz<float>(const float* S, const float* D, const float* u, float* v,
+                                        int n, long long E, cudaStream_t stream) {
+    return launch_ih_generic<float>(S, D, u, v, n, E, stream);
 }
 
 template <typename T>
@@ -79,10 +99,6 @@ cudaError_t launch_apply(const T* A, const T* B, const T* C, const T* u, T* v, i
     return launch_apply_generic<T>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream);
 }
 
-template cudaError_t launch_inv_helmholtz<double>(const double*, const double*, const double*,
-                                                  double*, int, long long, cudaStream_t);
-template cudaError_t launch_inv_helmholtz<float>(const float*, const float*, const float*, float*,
-                                                 int, long long, cudaStream_t);
 template cudaError_t launch_apply<double>(const double*, const double*, const double*,
                                           const double*, double*, int, int, int, int, int, int,
                                           long long, cudaStream_t);

@@ -53,6 +53,11 @@ int sm_count();
 bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
                         long long E, cudaStream_t stream, cudaError_t* err);
 
+// Tensor-path forward operator (fp64), same contract as try_launch_ih_dmma.
+bool try_launch_apply_dmma(const double* A, const double* B, const double* C, const double* u,
+                           double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
+                           cudaStream_t stream, cudaError_t* err);
+
 template <typename T>
 cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
                                  cudaStream_t stream);

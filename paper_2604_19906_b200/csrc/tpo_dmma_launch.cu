@@ -1,0 +1,83 @@
+// Instances and launchers of the tensor-path kernels.
+#include <cstdint>
+
+#include "dispatch.h"
+#include "tpo_dmma.cuh"
+
+namespace ekl {
+namespace {
+
+template <int N>
+cudaError_t launch_ih(const double* S, const double* D, const double* u, double* v, long long E,
+                      cudaStream_t stream) {
+    using C = dmma::IhCfg<N>;
+    cudaError_t err = cudaFuncSetAttribute(dmma::inv_helmholtz_dmma<N>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)C::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    int per_sm = 1;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dmma::inv_helmholtz_dmma<N>,
+                                                        C::kThreads, C::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long batches = (E + C::kBe - 1) / C::kBe;
+    long long grid = (long long)sm_count() * per_sm;
+    if (grid > batches) grid = batches;
+    dmma::inv_helmholtz_dmma<N><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    return cudaGetLastError();
+}
+
+template <int N0, int N1, int N2, int M0, int M1, int M2>
+cudaError_t launch_ap(const double* A, const double* B, const double* Cm, const double* u,
+                      double* v, long long E, cudaStream_t stream) {
+    using C = dmma::ApplyCfg<N0, N1, N2, M0, M1, M2>;
+    auto kernel = dmma::apply_dmma<N0, N1, N2, M0, M1, M2>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)C::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    int per_sm = 1;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, C::kThreads, C::kSmemBytes);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    const long long batches = (E + C::kBe - 1) / C::kBe;
+    long long grid = (long long)sm_count() * per_sm;
+    if (grid > batches) grid = batches;
+    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
+                        long long E, cudaStream_t stream, cudaError_t* err) {
+    // the bulk copy of u needs 16-byte aligned element addresses (8 n^3 is a multiple of 16
+    // for every even n)
+    if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+    switch (n) {
+        case 4: *err = launch_ih<4>(S, D, u, v, E, stream); return true;
+        case 6: *err = launch_ih<6>(S, D, u, v, E, stream); return true;
+        case 8: *err = launch_ih<8>(S, D, u, v, E, stream); return true;
+        case 10: *err = launch_ih<10>(S, D, u, v, E, stream); return true;
+        case 12: *err = launch_ih<12>(S, D, u, v, E, stream); return true;
+        case 14: *err = launch_ih<14>(S, D, u, v, E, stream); return true;
+        case 16: *err = launch_ih<16>(S, D, u, v, E, stream); return true;
+        default: return false;
+    }
+}
+
+bool try_launch_apply_dmma(const double* A, const double* B, const double* C, const double* u,
+                           double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
+                           cudaStream_t stream, cudaError_t* err) {
+    if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+    if (n0 == 8 && n1 == 8 && n2 == 8 && m0 == 12 && m1 == 12 && m2 == 12) {
+        *err = launch_ap<8, 8, 8, 12, 12, 12>(A, B, C, u, v, E, stream);
+        return true;
+    }
+    if (n0 == 12 && n1 == 12 && n2 == 12 && m0 == 8 && m1 == 8 && m2 == 8) {
+        *err = launch_ap<12, 12, 12, 8, 8, 8>(A, B, C, u, v, E, stream);
+        return true;
+    }
+    return false;
+}
+
+}  // namespace ekl

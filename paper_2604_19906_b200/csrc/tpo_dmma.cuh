@@ -15,8 +15,12 @@
 // to q*O + o = p1*(E2*O) + p2*O + o, which is again of that form for the next stage: it
 // contracts p1 over pencils (p2,o).  Three stages therefore cycle through the axes
 // i -> j -> k and end in the natural [i][j][k] order, so the input field is bulk-copied in
-// untouched and the pointwise factor and the output are addressed in their natural order.
-// With N = 2 or 6 (mod 8) every shared access of the stages is bank-conflict free.
+// plane by plane and the pointwise factor and the output are addressed in their natural
+// order.  Two paddings keep every shared access of the stages bank-conflict free: the row
+// stride (distance between consecutive p2) is 2 or 6 (mod 8) doubles, which spreads the
+// 4 pencil pairs x 4 output indices a half-warp stores, and the plane stride (distance
+// between consecutive contraction indices) is 4 (mod 8), which spreads the 4 contraction
+// indices x 4 pencils a half-warp loads.  For N = 14 (and 6, 10) both hold unpadded.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -94,29 +98,42 @@ __device__ __forceinline__ bool wait_bulk(uint64_t* bar, unsigned parity) {
     return true;
 }
 
-// One contraction stage for a batch of BE elements worked on by WARPS warps:
-// input [K][E1][E2] per element, output [E1][E2][O].
-template <int K_, int O_, int E1_, int E2_, int BE_, int WARPS_>
+// Smallest row stride >= o whose double-word count is 2 or 6 (mod 8).
+__host__ __device__ constexpr int pad_row(int o) {
+    return (o % 8 == 2 || o % 8 == 6) ? o : pad_row(o + 1);
+}
+// Smallest plane stride >= x that is 4 (mod 8).
+__host__ __device__ constexpr int pad_plane(int x) { return (x % 8 == 4) ? x : pad_plane(x + 1); }
+
+// One contraction stage for a batch of BE elements worked on by WARPS warps: input
+// [K][E1][E2] per element at  e*IN_ES + x*IN_PS + p1*IN_RS + p2,  output [E1][E2][O] at
+// e*OUT_ES + p1*OUT_PS + p2*OUT_RS + o  (dense global output: OUT_RS = O, OUT_PS = E2*O).
+template <int K_, int O_, int E1_, int E2_, int BE_, int WARPS_, int IN_RS_, int IN_PS_,
+          int IN_ES_, int OUT_RS_, int OUT_PS_, int OUT_ES_>
 struct Stage {
-    static constexpr int K = K_, O = O_, BE = BE_, WARPS = WARPS_;
-    static constexpr int kP = E1_ * E2_;                  // pencils per element
-    static constexpr int kIn = K * kP, kOut = O * kP;     // values per element
+    static constexpr int K = K_, O = O_, E1 = E1_, E2 = E2_, BE = BE_, WARPS = WARPS_;
+    static constexpr int IN_RS = IN_RS_, IN_PS = IN_PS_, IN_ES = IN_ES_;
+    static constexpr int OUT_RS = OUT_RS_, OUT_PS = OUT_PS_, OUT_ES = OUT_ES_;
+    static constexpr int kP = E1 * E2;                    // pencils per element
+    static constexpr int kIn = K * kP, kOut = O * kP;     // values per element (dense)
     static constexpr int kPencils = BE * kP;
     static constexpr int kTiles = (kPencils + 7) / 8;     // 8-pencil tiles, the last may be ragged
     static constexpr int kTilesPerWarp = (kTiles + WARPS - 1) / WARPS;
     static constexpr int kKSteps = (K + 3) / 4;
     static constexpr int kMTiles = (O + 7) / 8;
     static_assert(K >= 4, "contraction extent below one tensor step");
-    static_assert(kP % 2 == 0, "pencil pairs must not straddle elements");
+    static_assert(E2 % 2 == 0, "pencil pairs must share a row");
     // first contraction index of tensor step s; a last partial step overlaps the previous one
     __host__ __device__ static constexpr int k0(int s) { return (4 * s + 4 <= K) ? 4 * s : K - 4; }
 };
 
 // The operator matrix as this lane sees it: A[o][x], o = 8*mt + lane/4, x = k0(s) + lane%4.
-template <class SS>
-struct OpFrag {
-    double a[SS::kMTiles][SS::kKSteps];
+template <int MT, int KS>
+struct OpFragT {
+    double a[MT][KS];
 };
+template <class SS>
+using OpFrag = OpFragT<SS::kMTiles, SS::kKSteps>;
 
 // out_major: the matrix is stored [O][K] (A[o][x] = M[o*K + x]); otherwise [K][O], i.e. the
 // stage applies the transpose of the stored matrix (A[o][x] = M[x*O + o]).
@@ -145,7 +162,7 @@ __device__ __forceinline__ bool tile_live(int warp, int slot, int& t) {
     return slot < SS::kTilesPerWarp && t < SS::kTiles;
 }
 
-// The pointwise factor for the outputs this lane holds of tile slot `slot`.
+// The pointwise factor (dense, natural order) for the outputs this lane holds of tile `slot`.
 template <class SS>
 __device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2],
                                             const double* __restrict__ Db, int valid_pencils,
@@ -166,12 +183,12 @@ __device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2],
 
 // MODE 0: shared -> shared.  MODE 1: shared -> shared, times the pointwise factor (dfac
 // holds it for the warp's first tile on entry; later tiles are fetched one tile ahead from
-// Db).  MODE 2: shared -> global (gout).  `valid_pencils` masks a partly filled batch.
+// Db).  MODE 2: shared -> global (dense).  `valid_pencils` masks a partly filled batch.
 template <class SS, int MODE>
 __device__ __forceinline__ void run_stage(const double* __restrict__ in, double* __restrict__ out,
                                           const OpFrag<SS>& op, double (&dfac)[SS::kMTiles][2],
-                                          const double* __restrict__ Db, double* __restrict__ gout,
-                                          int valid_pencils, int warp, int lane) {
+                                          const double* __restrict__ Db, int valid_pencils,
+                                          int warp, int lane) {
     const int r = lane >> 2, kk = lane & 3;
 #pragma unroll
     for (int slot = 0; slot < SS::kTilesPerWarp; ++slot) {
@@ -181,10 +198,13 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
         int qb = 8 * t + r;
         if (qb >= SS::kPencils) qb = 0;                    // ragged last tile: any valid pencil
         const int eb = qb / SS::kP;
-        const double* src = in + eb * SS::kIn + (qb - eb * SS::kP) + kk * SS::kP;
+        const int pb = qb - eb * SS::kP;
+        const int pb1 = pb / SS::E2;
+        const double* src =
+            in + eb * SS::IN_ES + pb1 * SS::IN_RS + (pb - pb1 * SS::E2) + kk * SS::IN_PS;
         double b[SS::kKSteps];
 #pragma unroll
-        for (int s = 0; s < SS::kKSteps; ++s) b[s] = src[SS::k0(s) * SS::kP];
+        for (int s = 0; s < SS::kKSteps; ++s) b[s] = src[SS::k0(s) * SS::IN_PS];
         double dn[SS::kMTiles][2];
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp)
             load_factor<SS>(dn, Db, valid_pencils, warp, slot + 1, lane);
@@ -195,18 +215,21 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
 #pragma unroll
             for (int s = 0; s < SS::kKSteps; ++s) mma_f64(c[mt][0], c[mt][1], op.a[mt][s], b[s]);
         }
-        // this lane: output index o = 8*mt + r of pencils 8t + 2*kk + {0,1}; in a batch the
-        // output of element e, pencil q sits at e*kOut + q*O + o = (e*kP + q)*O + o
+        // this lane: output index o = 8*mt + r of pencils 8t + 2*kk + {0,1} (same row: E2 even)
         const int qs = 8 * t + 2 * kk;
         const bool ok = (MODE == 2) ? (qs < valid_pencils) : (qs < SS::kPencils);
         if (ok) {
-            double* dst = ((MODE == 2) ? gout : out) + (size_t)qs * SS::O;
+            const int es = qs / SS::kP;
+            const int ps = qs - es * SS::kP;
+            const int ps1 = ps / SS::E2;
+            double* dst = out + (size_t)es * SS::OUT_ES + ps1 * SS::OUT_PS +
+                          (ps - ps1 * SS::E2) * SS::OUT_RS;
 #pragma unroll
             for (int mt = 0; mt < SS::kMTiles; ++mt) {
                 const int o = 8 * mt + r;
                 if (o < SS::O) {
                     dst[o] = (MODE == 1) ? c[mt][0] * dfac[mt][0] : c[mt][0];
-                    dst[SS::O + o] = (MODE == 1) ? c[mt][1] * dfac[mt][1] : c[mt][1];
+                    dst[SS::OUT_RS + o] = (MODE == 1) ? c[mt][1] * dfac[mt][1] : c[mt][1];
                 }
             }
         }
@@ -217,6 +240,22 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
                 dfac[mt][1] = dn[mt][1];
             }
         }
+    }
+}
+
+// Thread 0: bring `cnt` dense elements of K planes x P values each from global memory into
+// the (possibly plane-padded) stage-input layout, all copies completing on `bar`.
+template <int K, int P, int PS, int ES>
+__device__ __forceinline__ void load_elements(double* dst, const double* src, int cnt,
+                                              uint64_t* bar) {
+    mbar_expect_tx(bar, (unsigned)(cnt * K * P * sizeof(double)));
+    if (PS == P && ES == K * P) {
+        bulk_load(dst, src, (unsigned)(cnt * K * P * sizeof(double)), bar);
+    } else {
+        for (int e = 0; e < cnt; ++e)
+            for (int x = 0; x < K; ++x)
+                bulk_load(dst + e * ES + x * PS, src + (size_t)(e * K + x) * P,
+                          (unsigned)(P * sizeof(double)), bar);
     }
 }
 
@@ -232,9 +271,15 @@ struct IhCfg {
                                   : (kTiles % 5 == 0) ? 5
                                   : (kTiles % 4 == 0) ? 4
                                                       : 8;
-    using SS = Stage<N, N, N, N, kBe, kWarps>;
+    // natural-order input planes, padded so that the first stage loads without conflicts
+    static constexpr int kPS0 = pad_plane(N * N), kES0 = N * kPS0;
+    // layout between stages
+    static constexpr int kRS = pad_row(N), kPS = pad_plane(N * kRS), kES = N * kPS;
+    using First = Stage<N, N, N, N, kBe, kWarps, N, kPS0, kES0, kRS, kPS, kES>;
+    using Mid = Stage<N, N, N, N, kBe, kWarps, kRS, kPS, kES, kRS, kPS, kES>;
+    using Last = Stage<N, N, N, N, kBe, kWarps, kRS, kPS, kES, N, N * N, N * N * N>;
     static constexpr int kThreads = 32 * kWarps;
-    static constexpr int kBufElems = kBe * N * N * N;
+    static constexpr int kBufElems = kBe * (kES0 > kES ? kES0 : kES);
     static constexpr size_t kSmemBytes = 2 * (size_t)kBufElems * sizeof(double) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
     static constexpr int kByWarps = 20 / kWarps;
@@ -249,8 +294,10 @@ __global__ void __launch_bounds__(IhCfg<N>::kThreads, IhCfg<N>::kCtasPerSm)
 inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, const double* u,
                    double* v, long long E) {
     using C = IhCfg<N>;
-    using SS = typename C::SS;
-    constexpr int kN3 = N * N * N;
+    using First = typename C::First;
+    using Mid = typename C::Mid;
+    using Last = typename C::Last;
+    constexpr int kN2 = N * N, kN3 = N * N * N;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     double* bufA = reinterpret_cast<double*>(smem_raw);
     double* bufB = bufA + C::kBufElems;
@@ -265,56 +312,56 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
 
-    auto batch_bytes = [&](long long b) {
+    auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
-        const long long cnt = (E - e0 < C::kBe) ? (E - e0) : C::kBe;
-        return (unsigned)(cnt * kN3 * sizeof(double));
+        return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
     long long batch = blockIdx.x;
-    if (threadIdx.x == 0 && batch < n_batches) {
-        mbar_expect_tx(bar, batch_bytes(batch));
-        bulk_load(bufA, u + batch * C::kBe * kN3, batch_bytes(batch), bar);
-    }
+    if (threadIdx.x == 0 && batch < n_batches)
+        load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3, batch_count(batch),
+                                                bar);
     unsigned parity = 0;
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
-        const int cnt = (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
-        const int valid = cnt * N * N;
+        const int cnt = batch_count(batch);
+        const int valid = cnt * kN2;
         const double* Db = D + e0 * kN3;
-        double* vb = v + e0 * kN3;
         const long long next = batch + gridDim.x;
         if (threadIdx.x == 0 && next < n_batches) {
-            bulk_prefetch_l2(u + next * C::kBe * kN3, batch_bytes(next));
-            bulk_prefetch_l2(D + next * C::kBe * kN3, batch_bytes(next));
+            const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(double));
+            bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
+            bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
         // forward stages apply S^T (t = sum_x S[x][o] in[x]); the fragments come from L1
-        OpFrag<SS> op;
-        load_op<SS>(op, S, false, lane);
-        double dfac[SS::kMTiles][2];
+        OpFrag<Mid> op;
+        load_op<Mid>(op, S, false, lane);
+        double dfac[Mid::kMTiles][2];
         if (!wait_bulk(bar, parity)) break;
         parity ^= 1u;
         // forward: contract i, j, k
-        run_stage<SS, 0>(bufA, bufB, op, dfac, nullptr, nullptr, valid, warp, lane);
+        run_stage<First, 0>(bufA, bufB, op, dfac, nullptr,
+                            valid, warp, lane);
         __syncthreads();
         // factor for this warp's first tile of the third stage: a whole stage hides the latency
-        load_factor<SS>(dfac, Db, valid, warp, 0, lane);
-        run_stage<SS, 0>(bufB, bufA, op, dfac, nullptr, nullptr, valid, warp, lane);
+        load_factor<Mid>(dfac, Db, valid, warp, 0, lane);
+        run_stage<Mid, 0>(bufB, bufA, op, dfac, nullptr, valid, warp, lane);
         __syncthreads();
-        run_stage<SS, 1>(bufA, bufB, op, dfac, Db, nullptr, valid, warp, lane);
+        run_stage<Mid, 1>(bufA, bufB, op, dfac, Db, valid, warp, lane);
         __syncthreads();
         // backward: contract i, j, k with S itself
-        load_op<SS>(op, S, true, lane);
-        run_stage<SS, 0>(bufB, bufA, op, dfac, nullptr, nullptr, valid, warp, lane);
+        load_op<Mid>(op, S, true, lane);
+        run_stage<Mid, 0>(bufB, bufA, op, dfac, nullptr, valid, warp, lane);
         __syncthreads();
-        run_stage<SS, 0>(bufA, bufB, op, dfac, nullptr, nullptr, valid, warp, lane);
+        run_stage<Mid, 0>(bufA, bufB, op, dfac, nullptr, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (threadIdx.x == 0 && next < n_batches) {
             fence_async_proxy();
-            mbar_expect_tx(bar, batch_bytes(next));
-            bulk_load(bufA, u + next * C::kBe * kN3, batch_bytes(next), bar);
+            load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
+                                                    batch_count(next), bar);
         }
-        run_stage<SS, 2>(bufB, nullptr, op, dfac, nullptr, vb, valid, warp, lane);
+        run_stage<Last, 2>(bufB, v + e0 * kN3, op, dfac,
+                           nullptr, valid, warp, lane);
         __syncthreads();
     }
 }
@@ -325,19 +372,25 @@ template <int N0, int N1, int N2, int M0, int M1, int M2>
 struct ApplyCfg {
     static constexpr int kBe = 2;
     static constexpr int kWarps = 4;
-    using S1 = Stage<N0, M0, N1, N2, kBe, kWarps>;     // [n0][n1][n2] -> [n1][n2][m0]
-    using S2 = Stage<N1, M1, N2, M0, kBe, kWarps>;     // [n1][n2][m0] -> [n2][m0][m1]
-    using S3 = Stage<N2, M2, M0, M1, kBe, kWarps>;     // [n2][m0][m1] -> [m0][m1][m2]
+    // u as it lands: [n0][n1*n2] with padded planes
+    static constexpr int kPS0 = pad_plane(N1 * N2), kES0 = N0 * kPS0;
+    // after the first stage: [n1][n2][m0]
+    static constexpr int kRS1 = pad_row(M0), kPS1 = pad_plane(N2 * kRS1), kES1 = N1 * kPS1;
+    // after the second stage: [n2][m0][m1]
+    static constexpr int kRS2 = pad_row(M1), kPS2 = pad_plane(M0 * kRS2), kES2 = N2 * kPS2;
+    using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
+    using S2 = Stage<N1, M1, N2, M0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
+    using S3 = Stage<N2, M2, M0, M1, kBe, kWarps, kRS2, kPS2, kES2, M2, M1 * M2, M0 * M1 * M2>;
     static constexpr int kThreads = 32 * kWarps;
-    static constexpr int kU = kBe * S1::kIn;           // landing buffer of u
-    static constexpr int kB = kBe * S1::kOut;          // first intermediate
-    static constexpr int kA = kBe * S2::kOut;          // second intermediate
+    static constexpr int kU = kBe * kES0;              // landing buffer of u
+    static constexpr int kB = kBe * kES1;              // first intermediate
+    static constexpr int kA = kBe * kES2;              // second intermediate
     static constexpr size_t kSmemBytes = (size_t)(kU + kB + kA) * sizeof(double) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
     static constexpr int kByWarps = 20 / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
-    static_assert((S1::kIn * sizeof(double)) % 16 == 0, "element size must allow bulk copies");
+    static_assert((N1 * N2) % 2 == 0, "planes must be a whole number of 16-byte units");
 };
 
 // v[e] = (A(x)B(x)C) u[e]; contraction order A, B, C (slowest axis first).
@@ -370,36 +423,33 @@ apply_dmma(const double* __restrict__ A, const double* __restrict__ B, const dou
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
-    auto batch_bytes = [&](long long b) {
+    auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
-        const long long cnt = (E - e0 < C::kBe) ? (E - e0) : C::kBe;
-        return (unsigned)(cnt * S1::kIn * sizeof(double));
+        return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
     long long batch = blockIdx.x;
-    if (threadIdx.x == 0 && batch < n_batches) {
-        mbar_expect_tx(bar, batch_bytes(batch));
-        bulk_load(bufU, u + batch * C::kBe * S1::kIn, batch_bytes(batch), bar);
-    }
+    if (threadIdx.x == 0 && batch < n_batches)
+        load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + batch * C::kBe * S1::kIn,
+                                                     batch_count(batch), bar);
     unsigned parity = 0;
     double none1[S1::kMTiles][2], none2[S2::kMTiles][2], none3[S3::kMTiles][2];
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
-        const int cnt = (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
+        const int cnt = batch_count(batch);
         const long long next = batch + gridDim.x;
         if (!wait_bulk(bar, parity)) break;
         parity ^= 1u;
-        run_stage<S1, 0>(bufU, bufB, opA, none1, nullptr, nullptr, cnt * S1::kP, warp, lane);
+        run_stage<S1, 0>(bufU, bufB, opA, none1, nullptr, cnt * S1::kP, warp, lane);
         __syncthreads();
         // the landing buffer is free: bring in the next batch under the remaining two stages
         if (threadIdx.x == 0 && next < n_batches) {
             fence_async_proxy();
-            mbar_expect_tx(bar, batch_bytes(next));
-            bulk_load(bufU, u + next * C::kBe * S1::kIn, batch_bytes(next), bar);
+            load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + next * C::kBe * S1::kIn,
+                                                         batch_count(next), bar);
         }
-        run_stage<S2, 0>(bufB, bufA, opB, none2, nullptr, nullptr, cnt * S2::kP, warp, lane);
+        run_stage<S2, 0>(bufB, bufA, opB, none2, nullptr, cnt * S2::kP, warp, lane);
         __syncthreads();
-        run_stage<S3, 2>(bufA, nullptr, opC, none3, nullptr, v + e0 * S3::kOut, cnt * S3::kP, warp,
-                         lane);
+        run_stage<S3, 2>(bufA, v + e0 * S3::kOut, opC, none3, nullptr, cnt * S3::kP, warp, lane);
         // the next batch's first stage writes bufB, which this batch no longer reads
     }
 }

@@ -42,6 +42,11 @@ SM_MAX_GHZ = 1.965
 FP64_PEAK_TFLOPS = SM_COUNT * FP64_LANES_PER_SM * 2 * SM_MAX_GHZ / 1e3
 HBM_FALLBACK_GBS = 6650.0
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per element of the operator
+# kernel, from the ncu captures summarised under profiles/ (taken on a smaller E of the same
+# kernel; traffic is proportional to the number of elements).  Workload index -> bytes.
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {3: 67195.0, 4: 16190.0}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -345,7 +350,10 @@ def main():
         roof = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
                 "frac": gbs / hbm_peak}
     roof.update({
-        "traffic": None,
+        "traffic": (NCU_TRAFFIC_BYTES_PER_ELEMENT[wl.index] * E
+                    if wl.index in NCU_TRAFFIC_BYTES_PER_ELEMENT and wl.dtype == "f64" else None),
+        "traffic_note": "bytes per launch: ncu dram read+write per element (profiles/) x E",
+        "algorithmic_bytes": bytes_launch, "algorithmic_flops": flops_launch,
         "kernel_ms": avg_launch_ms,
         "peak_source": ("alu: 148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz; hbm: "
                         f"MEASURED_PEAKS.json ({peak_src})"),

@@ -64,6 +64,9 @@ typedef enum {
  *
  * fp64.  `v == u` exactly (in place) is allowed; any other overlap of v with an
  * input is rejected.  1 <= n; n is limited by shared memory (n <= 24 for fp64).
+ * Even n from 4 to 16 with a 16-byte aligned u run on the FP64 tensor path (fastest);
+ * every other accepted case runs on a slower general kernel with the same results to
+ * rounding.
  */
 ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const double* u,
                                      double* v, int n, long long E, cudaStream_t stream);
@@ -176,6 +179,15 @@ int ekl_tpo_version(void);
 
 /* cudaError_t of the most recent EKL_TPO_ERR_CUDA returned on the calling thread. */
 int ekl_tpo_last_cuda_error(void);
+
+/*
+ * Device-side error flags since the last call of this function on the current device, and
+ * clears them; -1 if the query itself failed.  Bit 0: a kernel's bounded wait on one of its
+ * own bulk copies gave up (the kernel then stops early instead of hanging, and the output
+ * of that launch is not valid).  Not expected in practice; meant for health checks.
+ * SYNCHRONISES the device.  (Infrastructure: the paper has no counterpart.)
+ */
+int ekl_tpo_device_error_flags(void);
 
 /*
  * Measurement helper (no counterpart in the paper): enqueues `blocks` CTAs of 256

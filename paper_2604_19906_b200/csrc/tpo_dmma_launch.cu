@@ -81,3 +81,18 @@ bool try_launch_apply_dmma(const double* A, const double* B, const double* C, co
 }
 
 }  // namespace ekl
+
+// Reads (and clears) the flags device code raises when something that should never happen
+// did: bit 0 = a bounded wait on a bulk copy gave up, so the results of that launch are
+// not valid.  Synchronises the device.
+extern "C" int ekl_tpo_device_error_flags(void) {
+    int flag = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(&flag, ekl::dmma::g_bulk_wait_timeout, sizeof(int)) != cudaSuccess)
+        return -1;
+    if (flag) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(ekl::dmma::g_bulk_wait_timeout, &zero, sizeof(int));
+    }
+    return flag ? 1 : 0;
+}

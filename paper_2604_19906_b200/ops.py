@@ -13,7 +13,9 @@ import os
 
 import torch
 
-_LIBPATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libekl_tpo.so")
+# EKL_TPO_LIBRARY selects another build of the same library (A/B measurements)
+_LIBPATH = os.environ.get("EKL_TPO_LIBRARY") or os.path.join(
+    os.path.dirname(os.path.abspath(__file__)), "lib", "libekl_tpo.so")
 _lib = None
 
 STATUS_NAMES = {0: "EKL_TPO_OK", 1: "EKL_TPO_ERR_NULL", 2: "EKL_TPO_ERR_SHAPE",

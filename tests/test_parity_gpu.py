@@ -142,6 +142,31 @@ def test_element_permutation_and_batch_independence(env):
     assert torch.equal(shuf, full[p])
 
 
+@pytest.mark.parametrize("n", [8, 12, 14])
+def test_inv_helmholtz_unaligned_u_takes_the_general_kernel(env, n):
+    """u offset by one double is only 8-byte aligned: the tensor path (which bulk-copies u)
+    is skipped and the general kernel must give the same answer."""
+    torch = env["torch"]
+    E = 21
+    S, D, u = synth_ih(n, E, 31 + n)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    Sd, Dd = to_dev(env, S), to_dev(env, D)
+    store = torch.zeros(E * n ** 3 + 1, dtype=torch.float64, device=env["dev"])
+    ud = store[1:].view(E, n, n, n)
+    ud.copy_(to_dev(env, u))
+    assert ud.data_ptr() % 16 == 8
+    got = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud)
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+    aligned = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud.clone())
+    assert env["oracle"].rel_err_per_element(aligned.cpu().numpy(), want).max() <= TOL64
+
+
+def test_no_device_error_flags_after_all_this(env):
+    lib = env["ops"].library()
+    lib.ekl_tpo_device_error_flags.restype = __import__("ctypes").c_int
+    assert lib.ekl_tpo_device_error_flags() == 0
+
+
 # --------------------------------------------------------------------------- forward operator
 
 SHAPES = [((2, 3, 4), (5, 2, 3)), ((8, 8, 8), (12, 12, 12)), ((12, 12, 12), (8, 8, 8)),

@@ -308,6 +308,11 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
     const int lane = threadIdx.x & 31;
     const int warp = ((threadIdx.x >> 5) + blockIdx.x) % C::kWarps;
 
+    // forward stages apply S^T (t = sum_x S[x][o] in[x]), backward stages S itself
+    OpFrag<Mid> op, opb;
+    load_op<Mid>(op, S, false, lane);
+    load_op<Mid>(opb, S, true, lane);
+
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
@@ -332,9 +337,6 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
             bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
-        // forward stages apply S^T (t = sum_x S[x][o] in[x]); the fragments come from L1
-        OpFrag<Mid> op;
-        load_op<Mid>(op, S, false, lane);
         double dfac[Mid::kMTiles][2];
         if (!wait_bulk(bar, parity)) break;
         parity ^= 1u;
@@ -349,10 +351,9 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
         run_stage<Mid, 1>(bufA, bufB, op, dfac, Db, valid, warp, lane);
         __syncthreads();
         // backward: contract i, j, k with S itself
-        load_op<Mid>(op, S, true, lane);
-        run_stage<Mid, 0>(bufB, bufA, op, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0>(bufB, bufA, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 0>(bufA, bufB, op, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0>(bufA, bufB, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (threadIdx.x == 0 && next < n_batches) {
@@ -360,7 +361,7 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
             load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
                                                     batch_count(next), bar);
         }
-        run_stage<Last, 2>(bufB, v + e0 * kN3, op, dfac,
+        run_stage<Last, 2>(bufB, v + e0 * kN3, opb, dfac,
                            nullptr, valid, warp, lane);
         __syncthreads();
     }

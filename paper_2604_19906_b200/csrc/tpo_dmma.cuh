@@ -78,8 +78,14 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned b
         : "memory");
 }
 
+// L2 prefetch of a byte range; works in 16-byte granules, so a range that does not start on
+// one (odd extents, odd element index) is shrunk to the granules it fully contains.
 __device__ __forceinline__ void bulk_prefetch_l2(const void* src, unsigned bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+    const unsigned long long a = reinterpret_cast<unsigned long long>(src);
+    const unsigned lead = (unsigned)((16 - (a & 15)) & 15);
+    if (bytes < lead + 16) return;
+    const unsigned n = (bytes - lead) & ~15u;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(a + lead), "r"(n) : "memory");
 }
 
 __device__ __forceinline__ void fence_async_proxy() {
@@ -121,8 +127,9 @@ struct Stage {
     static constexpr int kTilesPerWarp = (kTiles + WARPS - 1) / WARPS;
     static constexpr int kKSteps = (K + 3) / 4;
     static constexpr int kMTiles = (O + 7) / 8;
+    // do the two neighbouring pencils a lane holds always share a row (and an element)?
+    static constexpr bool kPaired = (E2 % 2 == 0);
     static_assert(K >= 4, "contraction extent below one tensor step");
-    static_assert(E2 % 2 == 0, "pencil pairs must share a row");
     // first contraction index of tensor step s; a last partial step overlaps the previous one
     __host__ __device__ static constexpr int k0(int s) { return (4 * s + 4 <= K) ? 4 * s : K - 4; }
 };
@@ -175,9 +182,9 @@ __device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2],
 #pragma unroll
     for (int mt = 0; mt < SS::kMTiles; ++mt) {
         const int o = 8 * mt + r;
-        const bool ld = live && (qs < valid_pencils) && (o < SS::O);
-        d[mt][0] = ld ? __ldg(g + o) : 0.0;
-        d[mt][1] = ld ? __ldg(g + SS::O + o) : 0.0;
+        const bool ld = live && (o < SS::O);
+        d[mt][0] = (ld && qs < valid_pencils) ? __ldg(g + o) : 0.0;
+        d[mt][1] = (ld && qs + 1 < valid_pencils) ? __ldg(g + SS::O + o) : 0.0;
     }
 }
 
@@ -215,22 +222,23 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
 #pragma unroll
             for (int s = 0; s < SS::kKSteps; ++s) mma_f64(c[mt][0], c[mt][1], op.a[mt][s], b[s]);
         }
-        // this lane: output index o = 8*mt + r of pencils 8t + 2*kk + {0,1} (same row: E2 even)
+        // this lane: output index o = 8*mt + r of pencils 8t + 2*kk + {0,1}
         const int qs = 8 * t + 2 * kk;
-        const bool ok = (MODE == 2) ? (qs < valid_pencils) : (qs < SS::kPencils);
-        if (ok) {
-            const int es = qs / SS::kP;
-            const int ps = qs - es * SS::kP;
+        const int limit = (MODE == 2) ? valid_pencils : SS::kPencils;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            // with even rows the pair shares row and element, so one address serves both
+            const int q = SS::kPaired ? qs : qs + h;
+            if (q >= limit) continue;
+            const int es = q / SS::kP;
+            const int ps = q - es * SS::kP;
             const int ps1 = ps / SS::E2;
             double* dst = out + (size_t)es * SS::OUT_ES + ps1 * SS::OUT_PS +
-                          (ps - ps1 * SS::E2) * SS::OUT_RS;
+                          (ps - ps1 * SS::E2) * SS::OUT_RS + (SS::kPaired ? h * SS::OUT_RS : 0);
 #pragma unroll
             for (int mt = 0; mt < SS::kMTiles; ++mt) {
                 const int o = 8 * mt + r;
-                if (o < SS::O) {
-                    dst[o] = (MODE == 1) ? c[mt][0] * dfac[mt][0] : c[mt][0];
-                    dst[SS::OUT_RS + o] = (MODE == 1) ? c[mt][1] * dfac[mt][1] : c[mt][1];
-                }
+                if (o < SS::O) dst[o] = (MODE == 1) ? c[mt][h] * dfac[mt][h] : c[mt][h];
             }
         }
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp) {
@@ -259,11 +267,39 @@ __device__ __forceinline__ void load_elements(double* dst, const double* src, in
     }
 }
 
+// All threads: the same transfer with 8-byte asynchronous copies, for element sizes that are
+// not a multiple of 16 bytes (odd extents).  Completed by wait_copies().
+template <int K, int P, int PS, int ES>
+__device__ __forceinline__ void copy_elements(double* dst, const double* src, int cnt) {
+    const int total = cnt * K * P;
+    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+        const int e = idx / (K * P);
+        const int rem = idx - e * (K * P);
+        const int x = rem / P;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(
+                         smem_addr(dst + e * ES + x * PS + (rem - x * P))),
+                     "l"(src + idx)
+                     : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+__device__ __forceinline__ void wait_copies() {
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();
+}
+
 // ------------------------------------------------------------------ inverse Helmholtz
 
 template <int N>
 struct IhCfg {
-    static constexpr int kBe = (N >= 16) ? 1 : ((N <= 6) ? 4 : 2);      // elements per batch
+    // natural-order input planes, padded so that the first stage loads without conflicts
+    static constexpr int kPS0 = pad_plane(N * N), kES0 = N * kPS0;
+    // layout between stages
+    static constexpr int kRS = pad_row(N), kPS = pad_plane(N * kRS), kES = N * kPS;
+    static constexpr int kElemBuf = (kES0 > kES ? kES0 : kES);
+    // elements per batch: two (four for the smallest) unless that leaves room for one CTA only
+    static constexpr int kBe = (N <= 6) ? 4 : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
     static constexpr int kWarps = (N == 14)           ? 8
                                   : (kTiles % 8 == 0) ? 8
@@ -271,21 +307,19 @@ struct IhCfg {
                                   : (kTiles % 5 == 0) ? 5
                                   : (kTiles % 4 == 0) ? 4
                                                       : 8;
-    // natural-order input planes, padded so that the first stage loads without conflicts
-    static constexpr int kPS0 = pad_plane(N * N), kES0 = N * kPS0;
-    // layout between stages
-    static constexpr int kRS = pad_row(N), kPS = pad_plane(N * kRS), kES = N * kPS;
     using First = Stage<N, N, N, N, kBe, kWarps, N, kPS0, kES0, kRS, kPS, kES>;
     using Mid = Stage<N, N, N, N, kBe, kWarps, kRS, kPS, kES, kRS, kPS, kES>;
     using Last = Stage<N, N, N, N, kBe, kWarps, kRS, kPS, kES, N, N * N, N * N * N>;
     static constexpr int kThreads = 32 * kWarps;
-    static constexpr int kBufElems = kBe * (kES0 > kES ? kES0 : kES);
+    static constexpr int kBufElems = kBe * kElemBuf;
     static constexpr size_t kSmemBytes = 2 * (size_t)kBufElems * sizeof(double) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
     static constexpr int kByWarps = 20 / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
-    static_assert(N % 2 == 0 && N >= 4, "even N >= 4");
+    // bulk copies need 16-byte granules: even N; odd N uses 8-byte asynchronous copies
+    static constexpr bool kBulk = (N % 2 == 0);
+    static_assert(N >= 4, "N >= 4");
 };
 
 // v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])), u's element addresses 16-byte aligned.
@@ -322,9 +356,14 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
     long long batch = blockIdx.x;
-    if (threadIdx.x == 0 && batch < n_batches)
-        load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3, batch_count(batch),
-                                                bar);
+    if (batch < n_batches) {
+        if (!C::kBulk)
+            copy_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3,
+                                                    batch_count(batch));
+        else if (threadIdx.x == 0)
+            load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3,
+                                                    batch_count(batch), bar);
+    }
     unsigned parity = 0;
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
@@ -338,8 +377,12 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
             bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
         double dfac[Mid::kMTiles][2];
-        if (!wait_bulk(bar, parity)) break;
-        parity ^= 1u;
+        if (C::kBulk) {
+            if (!wait_bulk(bar, parity)) break;
+            parity ^= 1u;
+        } else {
+            wait_copies();
+        }
         // forward: contract i, j, k
         run_stage<First, 0>(bufA, bufB, op, dfac, nullptr,
                             valid, warp, lane);
@@ -356,10 +399,15 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
         run_stage<Mid, 0>(bufA, bufB, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
-        if (threadIdx.x == 0 && next < n_batches) {
-            fence_async_proxy();
-            load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
-                                                    batch_count(next), bar);
+        if (next < n_batches) {
+            if (!C::kBulk) {
+                copy_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
+                                                        batch_count(next));
+            } else if (threadIdx.x == 0) {
+                fence_async_proxy();
+                load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
+                                                        batch_count(next), bar);
+            }
         }
         run_stage<Last, 2>(bufB, v + e0 * kN3, opb, dfac,
                            nullptr, valid, warp, lane);

@@ -50,16 +50,22 @@ cudaError_t launch_ap(const double* A, const double* B, const double* Cm, const 
 
 bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
                         long long E, cudaStream_t stream, cudaError_t* err) {
-    // the bulk copy of u needs 16-byte aligned element addresses (8 n^3 is a multiple of 16
-    // for every even n)
-    if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+    // bulk copies of u (even n) need 16-byte aligned element addresses; odd n is copied in
+    // 8-byte units, and the L2 prefetches align themselves
+    if (n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     switch (n) {
         case 4: *err = launch_ih<4>(S, D, u, v, E, stream); return true;
+        case 5: *err = launch_ih<5>(S, D, u, v, E, stream); return true;
         case 6: *err = launch_ih<6>(S, D, u, v, E, stream); return true;
+        case 7: *err = launch_ih<7>(S, D, u, v, E, stream); return true;
         case 8: *err = launch_ih<8>(S, D, u, v, E, stream); return true;
+        case 9: *err = launch_ih<9>(S, D, u, v, E, stream); return true;
         case 10: *err = launch_ih<10>(S, D, u, v, E, stream); return true;
+        case 11: *err = launch_ih<11>(S, D, u, v, E, stream); return true;
         case 12: *err = launch_ih<12>(S, D, u, v, E, stream); return true;
+        case 13: *err = launch_ih<13>(S, D, u, v, E, stream); return true;
         case 14: *err = launch_ih<14>(S, D, u, v, E, stream); return true;
+        case 15: *err = launch_ih<15>(S, D, u, v, E, stream); return true;
         case 16: *err = launch_ih<16>(S, D, u, v, E, stream); return true;
         default: return false;
     }

@@ -161,6 +161,26 @@ def test_inv_helmholtz_unaligned_u_takes_the_general_kernel(env, n):
     assert env["oracle"].rel_err_per_element(aligned.cpu().numpy(), want).max() <= TOL64
 
 
+@pytest.mark.parametrize("n,E", [(5, 4099), (9, 2500), (13, 1201), (15, 999), (16, 700), (11, 1)])
+def test_inv_helmholtz_many_batches_per_cta(env, n, E):
+    """Enough elements that every persistent CTA loops over several batches and the last
+    batch is partly filled; u and D deliberately only 8-byte aligned for odd n."""
+    torch = env["torch"]
+    S, D, u = synth_ih(n, E, 7000 + n)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    off = 1 if n % 2 else 0
+    ubuf = torch.zeros(E * n ** 3 + 1, dtype=torch.float64, device=env["dev"])
+    dbuf = torch.zeros(E * n ** 3 + 1, dtype=torch.float64, device=env["dev"])
+    ud = ubuf[off:off + E * n ** 3].view(E, n, n, n)
+    dd = dbuf[off:off + E * n ** 3].view(E, n, n, n)
+    ud.copy_(to_dev(env, u))
+    dd.copy_(to_dev(env, D))
+    got = env["ops"].ekl_tpo_inv_helmholtz(to_dev(env, S), dd, ud)
+    torch.cuda.synchronize()
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy(), want)
+    assert err.max() <= TOL64, (n, E, err.max())
+
+
 def test_no_device_error_flags_after_all_this(env):
     lib = env["ops"].library()
     lib.ekl_tpo_device_error_flags.restype = __import__("ctypes").c_int

@@ -419,14 +419,16 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
 
 template <int N0, int N1, int N2, int M0, int M1, int M2>
 struct ApplyCfg {
-    static constexpr int kBe = 2;
-    static constexpr int kWarps = 4;
     // u as it lands: [n0][n1*n2] with padded planes
     static constexpr int kPS0 = pad_plane(N1 * N2), kES0 = N0 * kPS0;
     // after the first stage: [n1][n2][m0]
     static constexpr int kRS1 = pad_row(M0), kPS1 = pad_plane(N2 * kRS1), kES1 = N1 * kPS1;
     // after the second stage: [n2][m0][m1]
     static constexpr int kRS2 = pad_row(M1), kPS2 = pad_plane(M0 * kRS2), kES2 = N2 * kPS2;
+    // two elements per batch unless that leaves room for one CTA per SM only
+    static constexpr int kBe = ((kES0 + kES1 + kES2) * 2 * 8 <= 112 * 1024) ? 2 : 1;
+    // the last stage has the most tiles; give every warp at most about a dozen
+    static constexpr int kWarps = (kBe * M0 * M1 / 8 > 48) ? 8 : 4;
     using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
     using S2 = Stage<N1, M1, N2, M0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
     using S3 = Stage<N2, M2, M0, M1, kBe, kWarps, kRS2, kPS2, kES2, M2, M1 * M2, M0 * M1 * M2>;

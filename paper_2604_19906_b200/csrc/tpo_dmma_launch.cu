@@ -71,19 +71,42 @@ bool try_launch_ih_dmma(const double* S, const double* D, const double* u, doubl
     }
 }
 
+namespace {
+
+// cubic n -> m instances for even extents
+template <int N>
+bool apply_cubic_from(int m, const double* A, const double* B, const double* C, const double* u,
+                      double* v, long long E, cudaStream_t stream, cudaError_t* err) {
+    switch (m) {
+        case 4: *err = launch_ap<N, N, N, 4, 4, 4>(A, B, C, u, v, E, stream); return true;
+        case 6: *err = launch_ap<N, N, N, 6, 6, 6>(A, B, C, u, v, E, stream); return true;
+        case 8: *err = launch_ap<N, N, N, 8, 8, 8>(A, B, C, u, v, E, stream); return true;
+        case 10: *err = launch_ap<N, N, N, 10, 10, 10>(A, B, C, u, v, E, stream); return true;
+        case 12: *err = launch_ap<N, N, N, 12, 12, 12>(A, B, C, u, v, E, stream); return true;
+        case 14: *err = launch_ap<N, N, N, 14, 14, 14>(A, B, C, u, v, E, stream); return true;
+        case 16: *err = launch_ap<N, N, N, 16, 16, 16>(A, B, C, u, v, E, stream); return true;
+        default: return false;
+    }
+}
+
+}  // namespace
+
 bool try_launch_apply_dmma(const double* A, const double* B, const double* C, const double* u,
                            double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
                            cudaStream_t stream, cudaError_t* err) {
+    // u is bulk-copied plane by plane: 16-byte aligned element addresses
     if (reinterpret_cast<uintptr_t>(u) % 16) return false;
-    if (n0 == 8 && n1 == 8 && n2 == 8 && m0 == 12 && m1 == 12 && m2 == 12) {
-        *err = launch_ap<8, 8, 8, 12, 12, 12>(A, B, C, u, v, E, stream);
-        return true;
+    if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) return false;
+    switch (n0) {
+        case 4: return apply_cubic_from<4>(m0, A, B, C, u, v, E, stream, err);
+        case 6: return apply_cubic_from<6>(m0, A, B, C, u, v, E, stream, err);
+        case 8: return apply_cubic_from<8>(m0, A, B, C, u, v, E, stream, err);
+        case 10: return apply_cubic_from<10>(m0, A, B, C, u, v, E, stream, err);
+        case 12: return apply_cubic_from<12>(m0, A, B, C, u, v, E, stream, err);
+        case 14: return apply_cubic_from<14>(m0, A, B, C, u, v, E, stream, err);
+        case 16: return apply_cubic_from<16>(m0, A, B, C, u, v, E, stream, err);
+        default: return false;
     }
-    if (n0 == 12 && n1 == 12 && n2 == 12 && m0 == 8 && m1 == 8 && m2 == 8) {
-        *err = launch_ap<12, 12, 12, 8, 8, 8>(A, B, C, u, v, E, stream);
-        return true;
-    }
-    return false;
 }
 
 }  // namespace ekl

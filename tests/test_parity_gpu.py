@@ -206,6 +206,19 @@ def test_apply_f64(env, nn, mm, E):
     assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
 
 
+@pytest.mark.parametrize("n,m", [(4, 6), (6, 4), (10, 14), (14, 16), (16, 16), (16, 4), (12, 12),
+                                 (8, 8), (14, 10), (6, 16)])
+@pytest.mark.parametrize("E", [1, 2, 3, 257])
+def test_apply_f64_cubic_pairs_on_the_tensor_path(env, n, m, E):
+    g = rng(100 * n + m + E)
+    A, B, C = (g.standard_normal((m, n)) / np.sqrt(n) for _ in range(3))
+    u = g.uniform(-1, 1, (E, n, n, n))
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C, u)))
+    env["torch"].cuda.synchronize()
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+
+
 @pytest.mark.parametrize("nn,mm", SHAPES[:3])
 def test_apply_f32(env, nn, mm):
     g = rng(3)

@@ -48,15 +48,16 @@ void set_last_cuda_error(int err);
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
-// Tensor-path inverse Helmholtz (fp64).  Returns false if there is no instance for this n
-// or the pointers do not meet its alignment needs; otherwise launches and sets *err.
-bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
-                        long long E, cudaStream_t stream, cudaError_t* err);
-
-// Tensor-path forward operator (fp64), same contract as try_launch_ih_dmma.
-bool try_launch_apply_dmma(const double* A, const double* B, const double* C, const double* u,
-                           double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
-                           cudaStream_t stream, cudaError_t* err);
+// Tensor-path kernels (fp64 arithmetic; T is the type of the fields in memory).  Return false
+// if there is no instance for these extents or the pointers do not meet the alignment the
+// instance needs; otherwise launch and set *err.
+template <typename T>
+bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long long E,
+                        cudaStream_t stream, cudaError_t* err);
+template <typename T>
+bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
+                           int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,
+                           cudaError_t* err);
 
 template <typename T>
 cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,

@@ -79,36 +79,33 @@ static bool tuned_allowed() {
     return allowed;
 }
 
-template <>
-cudaError_t launch_inv_helmholtz<double>(const double* S, const double* D, const double* u,
-                                         double* v, int n, long long E, cudaStream_t stream) {
+template <typename T>
+cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
+                                 cudaStream_t stream) {
     cudaError_t err = cudaSuccess;
-    if (tuned_allowed() && try_launch_ih_dmma(S, D, u, v, n, E, stream, &err)) return err;
-    return launch_ih_generic<double>(S, D, u, v, n, E, stream);
+    if (tuned_allowed() && try_launch_ih_dmma<T>(S, D, u, v, n, E, stream, &err)) return err;
+    return launch_ih_generic<T>(S, D, u, v, n, E, stream);
 }
 
-template <>
-cudaError_t launch_inv_helmholtz<float>(const float* S, const float* D, const float* u, float* v,
-                                        int n, long long E, cudaStream_t stream) {
-    return launch_ih_generic<float>(S, D, u, v, n, E, stream);
-}
-
-template <>
-cudaError_t launch_apply<double>(const double* A, const double* B, const double* C,
-                                 const double* u, double* v, int n0, int n1, int n2, int m0, int m1,
-                                 int m2, long long E, cudaStream_t stream) {
+template <typename T>
+cudaError_t launch_apply(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
+                         int n2, int m0, int m1, int m2, long long E, cudaStream_t stream) {
     cudaError_t err = cudaSuccess;
     if (tuned_allowed() &&
-        try_launch_apply_dmma(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream, &err))
+        try_launch_apply_dmma<T>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream, &err))
         return err;
-    return launch_apply_generic<double>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream);
+    return launch_apply_generic<T>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream);
 }
 
-template <>
-cudaError_t launch_apply<float>(const float* A, const float* B, const float* C, const float* u,
-                                float* v, int n0, int n1, int n2, int m0, int m1, int m2,
-                                long long E, cudaStream_t stream) {
-    return launch_apply_generic<float>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream);
-}
+template cudaError_t launch_inv_helmholtz<double>(const double*, const double*, const double*,
+                                                  double*, int, long long, cudaStream_t);
+template cudaError_t launch_inv_helmholtz<float>(const float*, const float*, const float*, float*,
+                                                 int, long long, cudaStream_t);
+template cudaError_t launch_apply<double>(const double*, const double*, const double*,
+                                          const double*, double*, int, int, int, int, int, int,
+                                          long long, cudaStream_t);
+template cudaError_t launch_apply<float>(const float*, const float*, const float*, const float*,
+                                         float*, int, int, int, int, int, int, long long,
+                                         cudaStream_t);
 
 }  // namespace ekl

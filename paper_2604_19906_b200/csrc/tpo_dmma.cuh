@@ -144,8 +144,8 @@ using OpFrag = OpFragT<SS::kMTiles, SS::kKSteps>;
 
 // out_major: the matrix is stored [O][K] (A[o][x] = M[o*K + x]); otherwise [K][O], i.e. the
 // stage applies the transpose of the stored matrix (A[o][x] = M[x*O + o]).
-template <class SS>
-__device__ __forceinline__ void load_op(OpFrag<SS>& f, const double* __restrict__ M, bool out_major,
+template <class SS, typename T>
+__device__ __forceinline__ void load_op(OpFrag<SS>& f, const T* __restrict__ M, bool out_major,
                                         int lane) {
     const int r = lane >> 2, kk = lane & 3;
 #pragma unroll
@@ -157,7 +157,8 @@ __device__ __forceinline__ void load_op(OpFrag<SS>& f, const double* __restrict_
             const int x = SS::k0(s) + kk;
             const bool fresh = (s == 0) || (x >= SS::k0(s - 1) + 4);
             f.a[mt][s] =
-                (o < SS::O && fresh) ? __ldg(out_major ? M + o * SS::K + x : M + x * SS::O + o) : 0.0;
+                (o < SS::O && fresh) ? (double)__ldg(out_major ? M + o * SS::K + x : M + x * SS::O + o)
+                                     : 0.0;
         }
     }
 }
@@ -170,32 +171,33 @@ __device__ __forceinline__ bool tile_live(int warp, int slot, int& t) {
 }
 
 // The pointwise factor (dense, natural order) for the outputs this lane holds of tile `slot`.
-template <class SS>
-__device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2],
-                                            const double* __restrict__ Db, int valid_pencils,
-                                            int warp, int slot, int lane) {
+template <class SS, typename T>
+__device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2], const T* __restrict__ Db,
+                                            int valid_pencils, int warp, int slot, int lane) {
     const int r = lane >> 2, kk = lane & 3;
     int t;
     const bool live = tile_live<SS>(warp, slot, t);
     const int qs = 8 * t + 2 * kk;
-    const double* g = Db + (size_t)qs * SS::O;     // element e, pencil q: e*kOut + q*O
+    const T* g = Db + (size_t)qs * SS::O;          // element e, pencil q: e*kOut + q*O
 #pragma unroll
     for (int mt = 0; mt < SS::kMTiles; ++mt) {
         const int o = 8 * mt + r;
         const bool ld = live && (o < SS::O);
-        d[mt][0] = (ld && qs < valid_pencils) ? __ldg(g + o) : 0.0;
-        d[mt][1] = (ld && qs + 1 < valid_pencils) ? __ldg(g + SS::O + o) : 0.0;
+        d[mt][0] = (ld && qs < valid_pencils) ? (double)__ldg(g + o) : 0.0;
+        d[mt][1] = (ld && qs + 1 < valid_pencils) ? (double)__ldg(g + SS::O + o) : 0.0;
     }
 }
 
-// MODE 0: shared -> shared.  MODE 1: shared -> shared, times the pointwise factor (dfac
+// MODE 0: shared -> shared (out).  MODE 1: shared -> shared, times the pointwise factor (dfac
 // holds it for the warp's first tile on entry; later tiles are fetched one tile ahead from
-// Db).  MODE 2: shared -> global (dense).  `valid_pencils` masks a partly filled batch.
-template <class SS, int MODE>
+// Db).  MODE 2: shared -> global (gout, dense, converted to the I/O type T).
+// `valid_pencils` masks a partly filled batch.  All arithmetic is fp64 whatever T is.
+template <class SS, int MODE, typename T>
 __device__ __forceinline__ void run_stage(const double* __restrict__ in, double* __restrict__ out,
-                                          const OpFrag<SS>& op, double (&dfac)[SS::kMTiles][2],
-                                          const double* __restrict__ Db, int valid_pencils,
-                                          int warp, int lane) {
+                                          T* __restrict__ gout, const OpFrag<SS>& op,
+                                          double (&dfac)[SS::kMTiles][2],
+                                          const T* __restrict__ Db, int valid_pencils, int warp,
+                                          int lane) {
     const int r = lane >> 2, kk = lane & 3;
 #pragma unroll
     for (int slot = 0; slot < SS::kTilesPerWarp; ++slot) {
@@ -214,7 +216,7 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
         for (int s = 0; s < SS::kKSteps; ++s) b[s] = src[SS::k0(s) * SS::IN_PS];
         double dn[SS::kMTiles][2];
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp)
-            load_factor<SS>(dn, Db, valid_pencils, warp, slot + 1, lane);
+            load_factor<SS, T>(dn, Db, valid_pencils, warp, slot + 1, lane);
         double c[SS::kMTiles][2];
 #pragma unroll
         for (int mt = 0; mt < SS::kMTiles; ++mt) {
@@ -233,12 +235,17 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
             const int es = q / SS::kP;
             const int ps = q - es * SS::kP;
             const int ps1 = ps / SS::E2;
-            double* dst = out + (size_t)es * SS::OUT_ES + ps1 * SS::OUT_PS +
-                          (ps - ps1 * SS::E2) * SS::OUT_RS + (SS::kPaired ? h * SS::OUT_RS : 0);
+            const size_t off = (size_t)es * SS::OUT_ES + ps1 * SS::OUT_PS +
+                               (ps - ps1 * SS::E2) * SS::OUT_RS + (SS::kPaired ? h * SS::OUT_RS : 0);
 #pragma unroll
             for (int mt = 0; mt < SS::kMTiles; ++mt) {
                 const int o = 8 * mt + r;
-                if (o < SS::O) dst[o] = (MODE == 1) ? c[mt][h] * dfac[mt][h] : c[mt][h];
+                if (o < SS::O) {
+                    if (MODE == 2)
+                        gout[off + o] = (T)c[mt][h];
+                    else
+                        out[off + o] = (MODE == 1) ? c[mt][h] * dfac[mt][h] : c[mt][h];
+                }
             }
         }
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp) {
@@ -267,19 +274,25 @@ __device__ __forceinline__ void load_elements(double* dst, const double* src, in
     }
 }
 
-// All threads: the same transfer with 8-byte asynchronous copies, for element sizes that are
-// not a multiple of 16 bytes (odd extents).  Completed by wait_copies().
-template <int K, int P, int PS, int ES>
-__device__ __forceinline__ void copy_elements(double* dst, const double* src, int cnt) {
+// All threads: the same transfer without the bulk-copy engine, for element sizes that are not
+// a multiple of 16 bytes (odd extents: 8-byte asynchronous copies) and for single-precision
+// fields (plain loads, widened to fp64 on the way in).  Completed by wait_copies().
+template <int K, int P, int PS, int ES, typename T>
+__device__ __forceinline__ void copy_elements(double* dst, const T* __restrict__ src, int cnt) {
     const int total = cnt * K * P;
+#pragma unroll 4
     for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
         const int e = idx / (K * P);
         const int rem = idx - e * (K * P);
         const int x = rem / P;
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(
-                         smem_addr(dst + e * ES + x * PS + (rem - x * P))),
-                     "l"(src + idx)
-                     : "memory");
+        double* d = dst + e * ES + x * PS + (rem - x * P);
+        if (sizeof(T) == sizeof(double)) {
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_addr(d)),
+                         "l"(src + idx)
+                         : "memory");
+        } else {
+            *d = (double)__ldg(src + idx);
+        }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
@@ -302,6 +315,7 @@ struct IhCfg {
     static constexpr int kBe = (N <= 6) ? 4 : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
     static constexpr int kWarps = (N == 14)           ? 8
+                                  : (kTiles <= 16 && kTiles % 4 == 0) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6
                                   : (kTiles % 5 == 0) ? 5
@@ -322,12 +336,14 @@ struct IhCfg {
     static_assert(N >= 4, "N >= 4");
 };
 
-// v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])), u's element addresses 16-byte aligned.
-template <int N>
+// v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])).  T is the type of the fields in memory
+// (double: even N needs 16-byte aligned u; float: widened on load, rounded once on store).
+template <int N, typename T>
 __global__ void __launch_bounds__(IhCfg<N>::kThreads, IhCfg<N>::kCtasPerSm)
-inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, const double* u,
-                   double* v, long long E) {
+inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u, T* v,
+                   long long E) {
     using C = IhCfg<N>;
+    constexpr bool kBulk = C::kBulk && sizeof(T) == sizeof(double);
     using First = typename C::First;
     using Mid = typename C::Mid;
     using Last = typename C::Last;
@@ -344,8 +360,8 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
 
     // forward stages apply S^T (t = sum_x S[x][o] in[x]), backward stages S itself
     OpFrag<Mid> op, opb;
-    load_op<Mid>(op, S, false, lane);
-    load_op<Mid>(opb, S, true, lane);
+    load_op<Mid, T>(op, S, false, lane);
+    load_op<Mid, T>(opb, S, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
     if (threadIdx.x == 0) mbar_init(bar, 1);
@@ -357,60 +373,60 @@ inv_helmholtz_dmma(const double* __restrict__ S, const double* __restrict__ D, c
     };
     long long batch = blockIdx.x;
     if (batch < n_batches) {
-        if (!C::kBulk)
-            copy_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3,
+        if (!kBulk)
+            copy_elements<N, kN2, C::kPS0, C::kES0, T>(bufA, u + batch * C::kBe * kN3,
                                                     batch_count(batch));
         else if (threadIdx.x == 0)
-            load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3,
-                                                    batch_count(batch), bar);
+            load_elements<N, kN2, C::kPS0, C::kES0>(
+                bufA, reinterpret_cast<const double*>(u) + batch * C::kBe * kN3, batch_count(batch),
+                bar);
     }
     unsigned parity = 0;
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
         const int valid = cnt * kN2;
-        const double* Db = D + e0 * kN3;
+        const T* Db = D + e0 * kN3;
         const long long next = batch + gridDim.x;
         if (threadIdx.x == 0 && next < n_batches) {
-            const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(double));
+            const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(T));
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
             bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
         double dfac[Mid::kMTiles][2];
-        if (C::kBulk) {
+        if (kBulk) {
             if (!wait_bulk(bar, parity)) break;
             parity ^= 1u;
         } else {
             wait_copies();
         }
         // forward: contract i, j, k
-        run_stage<First, 0>(bufA, bufB, op, dfac, nullptr,
-                            valid, warp, lane);
+        run_stage<First, 0, T>(bufA, bufB, nullptr, op, dfac, nullptr, valid, warp, lane);
         __syncthreads();
         // factor for this warp's first tile of the third stage: a whole stage hides the latency
-        load_factor<Mid>(dfac, Db, valid, warp, 0, lane);
-        run_stage<Mid, 0>(bufB, bufA, op, dfac, nullptr, valid, warp, lane);
+        load_factor<Mid, T>(dfac, Db, valid, warp, 0, lane);
+        run_stage<Mid, 0, T>(bufB, bufA, nullptr, op, dfac, nullptr, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 1>(bufA, bufB, op, dfac, Db, valid, warp, lane);
+        run_stage<Mid, 1, T>(bufA, bufB, nullptr, op, dfac, Db, valid, warp, lane);
         __syncthreads();
         // backward: contract i, j, k with S itself
-        run_stage<Mid, 0>(bufB, bufA, opb, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0, T>(bufB, bufA, nullptr, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 0>(bufA, bufB, opb, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0, T>(bufA, bufB, nullptr, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (next < n_batches) {
-            if (!C::kBulk) {
-                copy_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
+            if (!kBulk) {
+                copy_elements<N, kN2, C::kPS0, C::kES0, T>(bufA, u + next * C::kBe * kN3,
                                                         batch_count(next));
             } else if (threadIdx.x == 0) {
                 fence_async_proxy();
-                load_elements<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
-                                                        batch_count(next), bar);
+                load_elements<N, kN2, C::kPS0, C::kES0>(
+                    bufA, reinterpret_cast<const double*>(u) + next * C::kBe * kN3,
+                    batch_count(next), bar);
             }
         }
-        run_stage<Last, 2>(bufB, v + e0 * kN3, opb, dfac,
-                           nullptr, valid, warp, lane);
+        run_stage<Last, 2, T>(bufB, nullptr, v + e0 * kN3, opb, dfac, nullptr, valid, warp, lane);
         __syncthreads();
     }
 }
@@ -445,12 +461,13 @@ struct ApplyCfg {
 };
 
 // v[e] = (A(x)B(x)C) u[e]; contraction order A, B, C (slowest axis first).
-template <int N0, int N1, int N2, int M0, int M1, int M2>
+template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
 __global__ void __launch_bounds__(ApplyCfg<N0, N1, N2, M0, M1, M2>::kThreads,
                                   ApplyCfg<N0, N1, N2, M0, M1, M2>::kCtasPerSm)
-apply_dmma(const double* __restrict__ A, const double* __restrict__ B, const double* __restrict__ Cm,
-           const double* __restrict__ u, double* __restrict__ v, long long E) {
+apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict__ Cm,
+           const T* __restrict__ u, T* __restrict__ v, long long E) {
     using C = ApplyCfg<N0, N1, N2, M0, M1, M2>;
+    constexpr bool kBulk = sizeof(T) == sizeof(double);
     using S1 = typename C::S1;
     using S2 = typename C::S2;
     using S3 = typename C::S3;
@@ -467,9 +484,9 @@ apply_dmma(const double* __restrict__ A, const double* __restrict__ B, const dou
     OpFrag<S1> opA;
     OpFrag<S2> opB;
     OpFrag<S3> opC;
-    load_op<S1>(opA, A, true, lane);
-    load_op<S2>(opB, B, true, lane);
-    load_op<S3>(opC, Cm, true, lane);
+    load_op<S1, T>(opA, A, true, lane);
+    load_op<S2, T>(opB, B, true, lane);
+    load_op<S3, T>(opC, Cm, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
     if (threadIdx.x == 0) mbar_init(bar, 1);
@@ -479,28 +496,37 @@ apply_dmma(const double* __restrict__ A, const double* __restrict__ B, const dou
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
     long long batch = blockIdx.x;
-    if (threadIdx.x == 0 && batch < n_batches)
-        load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + batch * C::kBe * S1::kIn,
-                                                     batch_count(batch), bar);
+    auto fetch = [&](long long b) {
+        if (!kBulk) {
+            copy_elements<N0, N1 * N2, C::kPS0, C::kES0, T>(bufU, u + b * C::kBe * S1::kIn,
+                                                            batch_count(b));
+        } else if (threadIdx.x == 0) {
+            fence_async_proxy();
+            load_elements<N0, N1 * N2, C::kPS0, C::kES0>(
+                bufU, reinterpret_cast<const double*>(u) + b * C::kBe * S1::kIn, batch_count(b), bar);
+        }
+    };
+    if (batch < n_batches) fetch(batch);
     unsigned parity = 0;
     double none1[S1::kMTiles][2], none2[S2::kMTiles][2], none3[S3::kMTiles][2];
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
         const long long next = batch + gridDim.x;
-        if (!wait_bulk(bar, parity)) break;
-        parity ^= 1u;
-        run_stage<S1, 0>(bufU, bufB, opA, none1, nullptr, cnt * S1::kP, warp, lane);
+        if (kBulk) {
+            if (!wait_bulk(bar, parity)) break;
+            parity ^= 1u;
+        } else {
+            wait_copies();
+        }
+        run_stage<S1, 0, T>(bufU, bufB, nullptr, opA, none1, nullptr, cnt * S1::kP, warp, lane);
         __syncthreads();
         // the landing buffer is free: bring in the next batch under the remaining two stages
-        if (threadIdx.x == 0 && next < n_batches) {
-            fence_async_proxy();
-            load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + next * C::kBe * S1::kIn,
-                                                         batch_count(next), bar);
-        }
-        run_stage<S2, 0>(bufB, bufA, opB, none2, nullptr, cnt * S2::kP, warp, lane);
+        if (next < n_batches) fetch(next);
+        run_stage<S2, 0, T>(bufB, bufA, nullptr, opB, none2, nullptr, cnt * S2::kP, warp, lane);
         __syncthreads();
-        run_stage<S3, 2>(bufA, v + e0 * S3::kOut, opC, none3, nullptr, cnt * S3::kP, warp, lane);
+        run_stage<S3, 2, T>(bufA, nullptr, v + e0 * S3::kOut, opC, none3, nullptr, cnt * S3::kP, warp,
+                            lane);
         // the next batch's first stage writes bufB, which this batch no longer reads
     }
 }

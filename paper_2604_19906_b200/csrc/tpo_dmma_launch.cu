@@ -7,38 +7,53 @@
 namespace ekl {
 namespace {
 
-template <int N>
-cudaError_t launch_ih(const double* S, const double* D, const double* u, double* v, long long E,
-                      cudaStream_t stream) {
+// Opts the kernel into its dynamic shared memory and asks how many CTAs fit on an SM; done
+// once per device and kernel (the answer is kept), so that repeated calls cost one launch.
+// Racing first calls compute the same value.
+// `cached` is the caller's per-kernel table (kernels of different shapes can share a
+// function-pointer type, so the table cannot live here).
+template <typename Kernel>
+cudaError_t ctas_per_sm(Kernel kernel, int threads, size_t smem, int (&cached)[64], int* per_sm) {
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cached[dev] == 0) {
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (err != cudaSuccess) return err;
+        int n = 1;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem);
+        if (err != cudaSuccess) return err;
+        cached[dev] = n < 1 ? 1 : n;
+    }
+    *per_sm = cached[dev];
+    return cudaSuccess;
+}
+
+template <int N, typename T>
+cudaError_t launch_ih(const T* S, const T* D, const T* u, T* v, long long E, cudaStream_t stream) {
     using C = dmma::IhCfg<N>;
-    cudaError_t err = cudaFuncSetAttribute(dmma::inv_helmholtz_dmma<N>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)C::kSmemBytes);
-    if (err != cudaSuccess) return err;
+    static int cached[64] = {0};
     int per_sm = 1;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dmma::inv_helmholtz_dmma<N>,
-                                                        C::kThreads, C::kSmemBytes);
+    cudaError_t err =
+        ctas_per_sm(dmma::inv_helmholtz_dmma<N, T>, C::kThreads, C::kSmemBytes, cached, &per_sm);
     if (err != cudaSuccess) return err;
-    if (per_sm < 1) per_sm = 1;
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
-    dmma::inv_helmholtz_dmma<N><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    dmma::inv_helmholtz_dmma<N, T><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
     return cudaGetLastError();
 }
 
-template <int N0, int N1, int N2, int M0, int M1, int M2>
-cudaError_t launch_ap(const double* A, const double* B, const double* Cm, const double* u,
-                      double* v, long long E, cudaStream_t stream) {
+template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
+cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, long long E,
+                      cudaStream_t stream) {
     using C = dmma::ApplyCfg<N0, N1, N2, M0, M1, M2>;
-    auto kernel = dmma::apply_dmma<N0, N1, N2, M0, M1, M2>;
-    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)C::kSmemBytes);
-    if (err != cudaSuccess) return err;
+    auto kernel = dmma::apply_dmma<N0, N1, N2, M0, M1, M2, T>;
+    static int cached[64] = {0};
     int per_sm = 1;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, C::kThreads, C::kSmemBytes);
+    cudaError_t err = ctas_per_sm(kernel, C::kThreads, C::kSmemBytes, cached, &per_sm);
     if (err != cudaSuccess) return err;
-    if (per_sm < 1) per_sm = 1;
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
@@ -48,25 +63,26 @@ cudaError_t launch_ap(const double* A, const double* B, const double* Cm, const 
 
 }  // namespace
 
-bool try_launch_ih_dmma(const double* S, const double* D, const double* u, double* v, int n,
-                        long long E, cudaStream_t stream, cudaError_t* err) {
-    // bulk copies of u (even n) need 16-byte aligned element addresses; odd n is copied in
-    // 8-byte units, and the L2 prefetches align themselves
-    if (n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
+template <typename T>
+bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long long E,
+                        cudaStream_t stream, cudaError_t* err) {
+    // bulk copies of u (fp64, even n) need 16-byte aligned element addresses; odd n and fp32
+    // fields are copied in element units, and the L2 prefetches align themselves
+    if (sizeof(T) == 8 && n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     switch (n) {
-        case 4: *err = launch_ih<4>(S, D, u, v, E, stream); return true;
-        case 5: *err = launch_ih<5>(S, D, u, v, E, stream); return true;
-        case 6: *err = launch_ih<6>(S, D, u, v, E, stream); return true;
-        case 7: *err = launch_ih<7>(S, D, u, v, E, stream); return true;
-        case 8: *err = launch_ih<8>(S, D, u, v, E, stream); return true;
-        case 9: *err = launch_ih<9>(S, D, u, v, E, stream); return true;
-        case 10: *err = launch_ih<10>(S, D, u, v, E, stream); return true;
-        case 11: *err = launch_ih<11>(S, D, u, v, E, stream); return true;
-        case 12: *err = launch_ih<12>(S, D, u, v, E, stream); return true;
-        case 13: *err = launch_ih<13>(S, D, u, v, E, stream); return true;
-        case 14: *err = launch_ih<14>(S, D, u, v, E, stream); return true;
-        case 15: *err = launch_ih<15>(S, D, u, v, E, stream); return true;
-        case 16: *err = launch_ih<16>(S, D, u, v, E, stream); return true;
+        case 4: *err = launch_ih<4, T>(S, D, u, v, E, stream); return true;
+        case 5: *err = launch_ih<5, T>(S, D, u, v, E, stream); return true;
+        case 6: *err = launch_ih<6, T>(S, D, u, v, E, stream); return true;
+        case 7: *err = launch_ih<7, T>(S, D, u, v, E, stream); return true;
+        case 8: *err = launch_ih<8, T>(S, D, u, v, E, stream); return true;
+        case 9: *err = launch_ih<9, T>(S, D, u, v, E, stream); return true;
+        case 10: *err = launch_ih<10, T>(S, D, u, v, E, stream); return true;
+        case 11: *err = launch_ih<11, T>(S, D, u, v, E, stream); return true;
+        case 12: *err = launch_ih<12, T>(S, D, u, v, E, stream); return true;
+        case 13: *err = launch_ih<13, T>(S, D, u, v, E, stream); return true;
+        case 14: *err = launch_ih<14, T>(S, D, u, v, E, stream); return true;
+        case 15: *err = launch_ih<15, T>(S, D, u, v, E, stream); return true;
+        case 16: *err = launch_ih<16, T>(S, D, u, v, E, stream); return true;
         default: return false;
     }
 }
@@ -74,40 +90,52 @@ bool try_launch_ih_dmma(const double* S, const double* D, const double* u, doubl
 namespace {
 
 // cubic n -> m instances for even extents
-template <int N>
-bool apply_cubic_from(int m, const double* A, const double* B, const double* C, const double* u,
-                      double* v, long long E, cudaStream_t stream, cudaError_t* err) {
+template <int N, typename T>
+bool apply_cubic_from(int m, const T* A, const T* B, const T* C, const T* u, T* v, long long E,
+                      cudaStream_t stream, cudaError_t* err) {
     switch (m) {
-        case 4: *err = launch_ap<N, N, N, 4, 4, 4>(A, B, C, u, v, E, stream); return true;
-        case 6: *err = launch_ap<N, N, N, 6, 6, 6>(A, B, C, u, v, E, stream); return true;
-        case 8: *err = launch_ap<N, N, N, 8, 8, 8>(A, B, C, u, v, E, stream); return true;
-        case 10: *err = launch_ap<N, N, N, 10, 10, 10>(A, B, C, u, v, E, stream); return true;
-        case 12: *err = launch_ap<N, N, N, 12, 12, 12>(A, B, C, u, v, E, stream); return true;
-        case 14: *err = launch_ap<N, N, N, 14, 14, 14>(A, B, C, u, v, E, stream); return true;
-        case 16: *err = launch_ap<N, N, N, 16, 16, 16>(A, B, C, u, v, E, stream); return true;
+        case 4: *err = launch_ap<N, N, N, 4, 4, 4, T>(A, B, C, u, v, E, stream); return true;
+        case 6: *err = launch_ap<N, N, N, 6, 6, 6, T>(A, B, C, u, v, E, stream); return true;
+        case 8: *err = launch_ap<N, N, N, 8, 8, 8, T>(A, B, C, u, v, E, stream); return true;
+        case 10: *err = launch_ap<N, N, N, 10, 10, 10, T>(A, B, C, u, v, E, stream); return true;
+        case 12: *err = launch_ap<N, N, N, 12, 12, 12, T>(A, B, C, u, v, E, stream); return true;
+        case 14: *err = launch_ap<N, N, N, 14, 14, 14, T>(A, B, C, u, v, E, stream); return true;
+        case 16: *err = launch_ap<N, N, N, 16, 16, 16, T>(A, B, C, u, v, E, stream); return true;
         default: return false;
     }
 }
 
 }  // namespace
 
-bool try_launch_apply_dmma(const double* A, const double* B, const double* C, const double* u,
-                           double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
-                           cudaStream_t stream, cudaError_t* err) {
-    // u is bulk-copied plane by plane: 16-byte aligned element addresses
-    if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+template <typename T>
+bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
+                           int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,
+                           cudaError_t* err) {
+    // fp64 u is bulk-copied plane by plane: 16-byte aligned element addresses
+    if (sizeof(T) == 8 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) return false;
     switch (n0) {
-        case 4: return apply_cubic_from<4>(m0, A, B, C, u, v, E, stream, err);
-        case 6: return apply_cubic_from<6>(m0, A, B, C, u, v, E, stream, err);
-        case 8: return apply_cubic_from<8>(m0, A, B, C, u, v, E, stream, err);
-        case 10: return apply_cubic_from<10>(m0, A, B, C, u, v, E, stream, err);
-        case 12: return apply_cubic_from<12>(m0, A, B, C, u, v, E, stream, err);
-        case 14: return apply_cubic_from<14>(m0, A, B, C, u, v, E, stream, err);
-        case 16: return apply_cubic_from<16>(m0, A, B, C, u, v, E, stream, err);
+        case 4: return apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err);
+        case 6: return apply_cubic_from<6, T>(m0, A, B, C, u, v, E, stream, err);
+        case 8: return apply_cubic_from<8, T>(m0, A, B, C, u, v, E, stream, err);
+        case 10: return apply_cubic_from<10, T>(m0, A, B, C, u, v, E, stream, err);
+        case 12: return apply_cubic_from<12, T>(m0, A, B, C, u, v, E, stream, err);
+        case 14: return apply_cubic_from<14, T>(m0, A, B, C, u, v, E, stream, err);
+        case 16: return apply_cubic_from<16, T>(m0, A, B, C, u, v, E, stream, err);
         default: return false;
     }
 }
+
+template bool try_launch_ih_dmma<double>(const double*, const double*, const double*, double*, int,
+                                         long long, cudaStream_t, cudaError_t*);
+template bool try_launch_ih_dmma<float>(const float*, const float*, const float*, float*, int,
+                                        long long, cudaStream_t, cudaError_t*);
+template bool try_launch_apply_dmma<double>(const double*, const double*, const double*,
+                                            const double*, double*, int, int, int, int, int, int,
+                                            long long, cudaStream_t, cudaError_t*);
+template bool try_launch_apply_dmma<float>(const float*, const float*, const float*, const float*,
+                                           float*, int, int, int, int, int, int, long long,
+                                           cudaStream_t, cudaError_t*);
 
 }  // namespace ekl
 

@@ -16,7 +16,9 @@ Operators (row-major arrays, element index slowest, see ``tpo_oracle.c``):
   lifted (sum-factorised) reductions of Section 5.2 of the paper.
 * ``tpo_apply(A, B, C, u)``: ``v_e = (A⊗B⊗C)·u_e``, rectangular factors, the
   operator family of Eq. 1.
-* ``*_bruteforce``: the same operators through the explicit Kronecker matrix.
+* ``convection(Dvq, Ivq, M, P)``: the volume integral of the convective flux, Eq. 1.
+* ``*_bruteforce``: the same operators through the explicit Kronecker matrix (or, for
+  ``convection``, the un-lifted sum of the paper's listing).
 * ``*_ld``: the same operators with every intermediate in ``long double``.
 """
 from __future__ import annotations
@@ -63,6 +65,10 @@ def _load():
         lib.oracle_tpo_apply_f64.argtypes = [dp, dp, dp, dp, dp, i, i, i, i, i, i, ll, i]
         lib.oracle_tpo_apply_bruteforce_f64.argtypes = [dp, dp, dp, dp, dp, i, i, i, i, i, i, ll]
         lib.oracle_tpo_apply_ld.argtypes = [dp, dp, dp, dp, dp, i, i, i, i, i, i, ll]
+        lib.oracle_convection_f64.argtypes = [dp, dp, dp, dp, dp, i, i, ll, i]
+        lib.oracle_convection_bruteforce_f64.argtypes = [dp, dp, dp, dp, dp, i, i, ll]
+        lib.oracle_convection_f64.restype = i
+        lib.oracle_convection_bruteforce_f64.restype = i
         for f in (lib.oracle_inv_helmholtz_f64, lib.oracle_inv_helmholtz_bruteforce_f64,
                   lib.oracle_inv_helmholtz_ld, lib.oracle_tpo_apply_f64,
                   lib.oracle_tpo_apply_bruteforce_f64, lib.oracle_tpo_apply_ld):
@@ -166,6 +172,42 @@ def tpo_apply_ld(A, B, C, u) -> np.ndarray:
                                          *nn, *mm, E):
         raise MemoryError("oracle scratch allocation failed")
     return v
+
+
+def _check_convection(Dvq, Ivq, M, P):
+    Dvq, Ivq, M, P = _f64(Dvq), _f64(Ivq), _f64(M), _f64(P)
+    if Dvq.ndim != 2 or Dvq.shape != Ivq.shape:
+        raise ValueError("Dvq and Ivq must both be [nv,nq]")
+    nv, nq = Dvq.shape
+    if M.ndim != 4 or M.shape[1:] != (nq, nq, nq):
+        raise ValueError("M must be [E,nq,nq,nq]")
+    E = M.shape[0]
+    if P.shape != (3, 3, E, nq, nq, nq):
+        raise ValueError("P must be [3,3,E,nq,nq,nq]")
+    return Dvq, Ivq, M, P, nq, nv, E
+
+
+def convection(Dvq, Ivq, M, P, threads: int = 0) -> np.ndarray:
+    """Volume integral of the convective flux (Eq. 1): for each component c and element e,
+    ``(I⊗I⊗D)(M∘P[c,0]) + (I⊗D⊗I)(M∘P[c,1]) + (D⊗I⊗I)(M∘P[c,2])``; returns F [3,E,nv,nv,nv]."""
+    Dvq, Ivq, M, P, nq, nv, E = _check_convection(Dvq, Ivq, M, P)
+    F = np.empty((3, E, nv, nv, nv), dtype=np.float64)
+    if E and _load().oracle_convection_f64(_ptr(Dvq), _ptr(Ivq), _ptr(M), _ptr(P), _ptr(F),
+                                           nq, nv, E, int(threads)):
+        raise MemoryError("oracle scratch allocation failed")
+    return F
+
+
+def convection_bruteforce(Dvq, Ivq, M, P) -> np.ndarray:
+    """The same operator as one un-lifted sum over (l,m,n) per output (tiny sizes only)."""
+    Dvq, Ivq, M, P, nq, nv, E = _check_convection(Dvq, Ivq, M, P)
+    if nq > 6 or nv > 6:
+        raise ValueError("brute force is meant for tiny shapes")
+    F = np.empty((3, E, nv, nv, nv), dtype=np.float64)
+    if E:
+        _load().oracle_convection_bruteforce_f64(_ptr(Dvq), _ptr(Ivq), _ptr(M), _ptr(P), _ptr(F),
+                                                 nq, nv, E)
+    return F
 
 
 def rel_err_per_element(v, v_ref) -> np.ndarray:

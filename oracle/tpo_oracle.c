@@ -161,6 +161,86 @@ int oracle_inv_helmholtz_f64(const double *S, const double *D, const double *u,
     return fail ? -1 : 0;
 }
 
+/*
+ * Volume integral of the convective flux (Eq. 1 of the paper and its one-statement
+ * listing), sum-factorised term by term:
+ *
+ *   F[c,e] = (I (x) I (x) D) (M[e] o P[c,0,e]) + (I (x) D (x) I) (M[e] o P[c,1,e])
+ *          + (D (x) I (x) I) (M[e] o P[c,2,e]),          c = 0,1,2
+ *
+ * with the first Kronecker factor on the slowest in-element axis (k/n in the listing's
+ * index names) and the last on the fastest (i/l).  Dvq, Ivq: [nv,nq];  M: [E,nq,nq,nq];
+ * P: [3,3,E,nq,nq,nq];  F: [3,E,nv,nv,nv].
+ */
+int oracle_convection_f64(const double *Dvq, const double *Ivq, const double *M, const double *P,
+                          double *F, int nq, int nv, long long E, int threads)
+{
+    const size_t q3 = (size_t)nq * nq * nq, v3 = (size_t)nv * nv * nv;
+    int fail = 0;
+    threads = pick_threads(threads);
+#pragma omp parallel num_threads(threads)
+    {
+        const size_t np = (size_t)nq * nq * nv, nqq = (size_t)nq * nv * nv;
+        double *w = (double *)malloc((q3 + np + nqq + v3 + 1) * sizeof(double));
+        if (!w) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+            double *x = w, *p = x + q3, *q = p + np, *t = q + nqq;
+#pragma omp for schedule(static) collapse(2)
+            for (int c = 0; c < 3; ++c)
+                for (long long e = 0; e < E; ++e) {
+                    double *Fe = F + ((size_t)c * E + e) * v3;
+                    for (size_t y = 0; y < v3; ++y) Fe[y] = 0.0;
+                    for (int d = 0; d < 3; ++d) {
+                        const double *Pd = P + (((size_t)c * 3 + d) * E + e) * q3;
+                        for (size_t y = 0; y < q3; ++y) x[y] = M[(size_t)e * q3 + y] * Pd[y];
+                        /* the derivative matrix sits on the fastest axis for d = 0, the
+                         * middle one for d = 1, the slowest for d = 2 */
+                        const double *A = (d == 2) ? Dvq : Ivq;
+                        const double *B = (d == 1) ? Dvq : Ivq;
+                        const double *C = (d == 0) ? Dvq : Ivq;
+                        apply_one(A, B, C, x, t, p, q, nq, nq, nq, nv, nv, nv);
+                        for (size_t y = 0; y < v3; ++y) Fe[y] = Fe[y] + t[y];
+                    }
+                }
+        }
+        free(w);
+    }
+    return fail ? -1 : 0;
+}
+
+/* The same operator as the listing states it: one un-lifted sum over (l,m,n) per output. */
+int oracle_convection_bruteforce_f64(const double *Dvq, const double *Ivq, const double *M,
+                                     const double *P, double *F, int nq, int nv, long long E)
+{
+    const size_t q3 = (size_t)nq * nq * nq;
+    for (int c = 0; c < 3; ++c)
+        for (long long e = 0; e < E; ++e)
+            for (int k = 0; k < nv; ++k)
+                for (int j = 0; j < nv; ++j)
+                    for (int i = 0; i < nv; ++i) {
+                        double s = 0.0;
+                        for (int n = 0; n < nq; ++n)
+                            for (int m = 0; m < nq; ++m)
+                                for (int l = 0; l < nq; ++l) {
+                                    const size_t y = ((size_t)n * nq + m) * nq + l;
+                                    const double Me = M[(size_t)e * q3 + y];
+                                    const double *Pc = P + ((size_t)c * 3 * E + e) * q3 + y;
+                                    s = s + Dvq[i * nq + l] * Ivq[j * nq + m] * Ivq[k * nq + n] *
+                                                Me * Pc[0]
+                                          + Ivq[i * nq + l] * Dvq[j * nq + m] * Ivq[k * nq + n] *
+                                                Me * Pc[(size_t)E * q3]
+                                          + Ivq[i * nq + l] * Ivq[j * nq + m] * Dvq[k * nq + n] *
+                                                Me * Pc[2 * (size_t)E * q3];
+                                }
+                        F[(((size_t)c * E + e) * nv + k) * nv * nv + (size_t)j * nv + i] = s;
+                    }
+    return 0;
+}
+
 /* ---- the un-lifted definition ------------------------------------------- */
 
 /* K[(i m1 + j) m2 + k , (l n1 + m) n2 + n] = A[i,l] B[j,m] C[k,n]           */

@@ -242,3 +242,57 @@ def test_flop_accounting_matches_the_lifting_claim():
     assert CONFIGS[4].flops_per_element == 58368
     assert CONFIGS[4].bytes_per_element == 17920
     assert CONFIGS[3].bytes_per_element == 65856
+
+
+# ------------------------------------------------------------------ convective flux (Eq. 1)
+
+def ref_convection_einsum(Dvq, Ivq, M, P):
+    """The paper's one-statement form, index names as printed: F[c,e,k,j,i] with (l,m,n)
+    summed, D on the (i,l) pair for direction 0, on (j,m) for 1, on (k,n) for 2."""
+    out = []
+    for c in range(3):
+        t = (np.einsum("il,jm,kn,enml,enml->ekji", Dvq, Ivq, Ivq, M, P[c, 0])
+             + np.einsum("il,jm,kn,enml,enml->ekji", Ivq, Dvq, Ivq, M, P[c, 1])
+             + np.einsum("il,jm,kn,enml,enml->ekji", Ivq, Ivq, Dvq, M, P[c, 2]))
+        out.append(t)
+    return np.stack(out)
+
+
+@pytest.mark.parametrize("nq,nv", [(3, 2), (4, 4), (5, 3), (2, 5), (12, 8)])
+def test_convection_matches_the_printed_statement(nq, nv):
+    g = rng(400 + nq * 10 + nv)
+    E = 3
+    Dvq, Ivq = g.standard_normal((2, nv, nq))
+    M = g.uniform(0.5, 1.5, (E, nq, nq, nq))
+    P = g.uniform(-1, 1, (3, 3, E, nq, nq, nq))
+    F = oracle.convection(Dvq, Ivq, M, P)
+    ref = ref_convection_einsum(Dvq, Ivq, M, P)
+    assert F.shape == (3, E, nv, nv, nv)
+    assert relmax(F.reshape(3 * E, nv, nv, nv), ref.reshape(3 * E, nv, nv, nv)) < 1e-13
+    if nq <= 6 and nv <= 6:
+        bf = oracle.convection_bruteforce(Dvq, Ivq, M, P)
+        assert relmax(bf.reshape(3 * E, nv, nv, nv), ref.reshape(3 * E, nv, nv, nv)) < 1e-13
+
+
+def test_convection_special_cases_and_planted_mistakes():
+    g = rng(17)
+    nq, nv, E = 4, 3, 2
+    Dvq, Ivq = g.standard_normal((2, nv, nq))
+    M = g.uniform(0.5, 1.5, (E, nq, nq, nq))
+    P = g.uniform(-1, 1, (3, 3, E, nq, nq, nq))
+    ref = ref_convection_einsum(Dvq, Ivq, M, P).reshape(3 * E, nv, nv, nv)
+    flat = lambda F: F.reshape(3 * E, nv, nv, nv)
+    # each direction alone is one forward operator with D on its own axis (M = 1)
+    ones = np.ones_like(M)
+    for d, (A, B, C) in enumerate([(Ivq, Ivq, Dvq), (Ivq, Dvq, Ivq), (Dvq, Ivq, Ivq)]):
+        Pd = np.zeros_like(P)
+        Pd[:, d] = P[:, d]
+        want = np.stack([oracle.tpo_apply(A, B, C, P[c, d]) for c in range(3)])
+        assert relmax(flat(oracle.convection(Dvq, Ivq, ones, Pd)), flat(want)) < 1e-13
+    # D = 0 kills everything; M scales linearly
+    assert np.all(oracle.convection(np.zeros_like(Dvq), Ivq, M, P) == 0.0)
+    assert relmax(flat(oracle.convection(Dvq, Ivq, 2.0 * M, P)), 2.0 * ref) < 1e-13
+    # planted slips are seen by the reference
+    assert relmax(flat(oracle.convection(Ivq, Dvq, M, P)), ref) > 1e-3          # D and I swapped
+    assert relmax(flat(oracle.convection(Dvq, Ivq, M, P[:, ::-1].copy())), ref) > 1e-3  # directions
+    assert relmax(flat(oracle.convection(Dvq, Ivq, ones, P)), ref) > 1e-3       # dropped M

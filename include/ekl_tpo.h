@@ -85,6 +85,29 @@ ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
                              int n0, int n1, int n2, int m0, int m1, int m2,
                              long long E, cudaStream_t stream);
 
+/*
+ * Volume integral of the convective flux (Eq. 1 of the paper; the `convection` kernel,
+ * the one-statement listing next to it), for the three components c = 0,1,2:
+ *
+ *     F[c,e] = (I (x) I (x) D) . (M[e] o P[c,0,e]) + (I (x) D (x) I) . (M[e] o P[c,1,e])
+ *            + (D (x) I (x) I) . (M[e] o P[c,2,e])
+ *
+ *   Dvq, Ivq [nv,nq]   differentiation / interpolation from quadrature to volume points
+ *   M   [E,nq,nq,nq]   pointwise factor shared by the components and directions
+ *   P   [3,3,E,nq,nq,nq]   fluxes, indexed [component][direction][element]...
+ *   F   [3,E,nv,nv,nv]
+ *
+ * i.e. F[c,e,k,j,i] = sum_{l,m,n} ( D[i,l] I[j,m] I[k,n] P[c,0,e,n,m,l] + I[i,l] D[j,m] I[k,n]
+ * P[c,1,e,n,m,l] + I[i,l] I[j,m] D[k,n] P[c,2,e,n,m,l] ) M[e,n,m,l]: the derivative acts on the
+ * fastest axis for direction 0 and on the slowest for direction 2.  fp64.  M and P must be
+ * 16-byte aligned (EKL_TPO_ERR_ALIGN otherwise); F must not overlap any input.  Available
+ * for (nq,nv) in {(4,4),(6,4),(6,6),(8,4),(8,6),(8,8),(10,8),(10,10),(12,8),(12,10),(12,12),
+ * (14,12)}; other extents return EKL_TPO_ERR_UNSUPPORTED.
+ */
+ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const double* M,
+                                  const double* P, double* F, int nq, int nv, long long E,
+                                  cudaStream_t stream);
+
 /* Single-precision twins of the two operators above (same layout and rules). */
 ekl_tpo_status ekl_tpo_inv_helmholtz_f32(const float* S, const float* D, const float* u,
                                          float* v, int n, long long E, cudaStream_t stream);

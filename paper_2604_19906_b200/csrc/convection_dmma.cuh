@@ -1,0 +1,190 @@
+// Volume integral of the convective flux (Eq. 1 of the paper) on the FP64 tensor path.
+//
+//   F[c,e] = (I(x)I(x)D)(M[e] o P[c,0,e]) + (I(x)D(x)I)(M[e] o P[c,1,e]) + (D(x)I(x)I)(M[e] o P[c,2,e])
+//
+// with the first Kronecker factor on the slowest in-element axis.  Sum-factorised with the
+// shared contractions merged: with x_d = M o P_d,
+//   stage 1 (slowest axis):  t0 = I x0,  t1 = I x1,  t2 = D x2
+//   stage 2 (middle axis):   w0 = I t0,  w12 = D t1 + I t2
+//   stage 3 (fastest axis):  F  = D w0 + I w12
+// The two-term stages accumulate both products in the same tensor accumulators, so no
+// element-wise add and no third intermediate exist.  Stages use the machinery of
+// tpo_dmma.cuh (operator as register A fragments, 8-pencil B tiles from shared memory,
+// cycling layouts with conflict-free padding).  M is applied while the B fragments of the
+// first stage are read.  One CTA works on one element at a time: M[e] is fetched once and
+// serves the three components; the P fields of the next component are bulk-copied under
+// stages 2 and 3 of the current one.
+#pragma once
+#include "tpo_dmma.cuh"
+
+namespace ekl {
+namespace dmma {
+
+template <int NQ, int NV>
+struct ConvCfg {
+    static constexpr int kWarps = 8;
+    static constexpr int kThreads = 32 * kWarps;
+    // fields as they land: [n][(m,l)], padded planes
+    static constexpr int kPS0 = pad_plane(NQ * NQ), kES0 = NQ * kPS0;
+    // after stage 1: [m][l][n']
+    static constexpr int kRS1 = pad_row(NV), kPS1 = pad_plane(NQ * kRS1), kES1 = NQ * kPS1;
+    // after stage 2: [l][n'][m']
+    static constexpr int kRS2 = pad_row(NV), kPS2 = pad_plane(NV * kRS2), kES2 = NQ * kPS2;
+    using S1 = Stage<NQ, NV, NQ, NQ, 1, kWarps, NQ, kPS0, kES0, kRS1, kPS1, kES1>;
+    using S2 = Stage<NQ, NV, NQ, NV, 1, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
+    using S3 = Stage<NQ, NV, NV, NV, 1, kWarps, kRS2, kPS2, kES2, NV, NV * NV, NV * NV * NV>;
+    // shared memory: M, three P fields, three stage-1 outputs, two stage-2 outputs
+    static constexpr int kDoubles = 4 * kES0 + 3 * kES1 + 2 * kES2;
+    static constexpr size_t kSmemBytes = (size_t)kDoubles * sizeof(double) + 16;
+    static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
+    static constexpr int kCtasPerSm = kBySmem < 1 ? 1 : (kBySmem > 2 ? 2 : kBySmem);
+    static_assert(NQ % 2 == 0 && NV % 2 == 0, "even extents (bulk copies, paired stores)");
+    static_assert(S1::kMTiles == S2::kMTiles && S1::kKSteps == S3::kKSteps, "one fragment shape");
+};
+
+// Accumulate one (operator, input) product of tile t into c; the input may be scaled
+// entry-wise by `scale` (same layout as `in`).
+template <class SS, bool SCALE>
+__device__ __forceinline__ void tile_accumulate(double (&c)[SS::kMTiles][2], const OpFrag<SS>& op,
+                                                const double* __restrict__ in,
+                                                const double* __restrict__ scale, int t, int lane) {
+    const int r = lane >> 2, kk = lane & 3;
+    int qb = 8 * t + r;
+    if (qb >= SS::kPencils) qb = 0;
+    const int pb1 = qb / SS::E2;
+    const int off = pb1 * SS::IN_RS + (qb - pb1 * SS::E2) + kk * SS::IN_PS;
+    double b[SS::kKSteps];
+#pragma unroll
+    for (int s = 0; s < SS::kKSteps; ++s) {
+        b[s] = in[off + SS::k0(s) * SS::IN_PS];
+        if (SCALE) b[s] *= scale[off + SS::k0(s) * SS::IN_PS];
+    }
+#pragma unroll
+    for (int mt = 0; mt < SS::kMTiles; ++mt)
+#pragma unroll
+        for (int s = 0; s < SS::kKSteps; ++s) mma_f64(c[mt][0], c[mt][1], op.a[mt][s], b[s]);
+}
+
+// Write the accumulators of tile t to the stage's output layout (`out` in shared memory, or
+// dense global memory when TO_GLOBAL).
+template <class SS, bool TO_GLOBAL>
+__device__ __forceinline__ void tile_store(const double (&c)[SS::kMTiles][2], double* out, int t,
+                                           int lane) {
+    const int r = lane >> 2, kk = lane & 3;
+    const int qs = 8 * t + 2 * kk;
+    if (qs >= SS::kPencils) return;
+    const int ps1 = qs / SS::E2;
+    double* dst = out + ps1 * SS::OUT_PS + (qs - ps1 * SS::E2) * SS::OUT_RS;
+#pragma unroll
+    for (int mt = 0; mt < SS::kMTiles; ++mt) {
+        const int o = 8 * mt + r;
+        if (o < SS::O) {
+            dst[o] = c[mt][0];
+            dst[SS::OUT_RS + o] = c[mt][1];
+        }
+    }
+}
+
+template <int NQ, int NV>
+__global__ void __launch_bounds__(ConvCfg<NQ, NV>::kThreads, ConvCfg<NQ, NV>::kCtasPerSm)
+convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
+                const double* __restrict__ M, const double* __restrict__ P, double* __restrict__ F,
+                long long E) {
+    using C = ConvCfg<NQ, NV>;
+    using S1 = typename C::S1;
+    using S2 = typename C::S2;
+    using S3 = typename C::S3;
+    constexpr int kQ3 = NQ * NQ * NQ, kV3 = NV * NV * NV;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    double* sM = reinterpret_cast<double*>(smem_raw);
+    double* sX = sM + C::kES0;                  // three P fields
+    double* sT = sX + 3 * C::kES0;              // t0, t1, t2
+    double* sW = sT + 3 * C::kES1;              // w0, w12
+    uint64_t* bar = reinterpret_cast<uint64_t*>(sW + 2 * C::kES2);
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // both operators have the same shape in every stage ([nv,nq], output index major)
+    OpFrag<S1> opI, opD;
+    load_op<S1, double>(opI, Ivq, true, lane);
+    load_op<S1, double>(opD, Dvq, true, lane);
+
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    __syncthreads();
+
+    // thread 0: bulk-copy the P fields of (c, e) -- and M[e] when asked -- plane by plane
+    auto fetch = [&](int c, long long e, bool with_m) {
+        const unsigned field = (unsigned)(kQ3 * sizeof(double));
+        mbar_expect_tx(bar, (with_m ? 4u : 3u) * field);
+        if (with_m)
+            for (int x = 0; x < NQ; ++x)
+                bulk_load(sM + x * C::kPS0, M + (size_t)e * kQ3 + x * NQ * NQ,
+                          (unsigned)(NQ * NQ * sizeof(double)), bar);
+        for (int d = 0; d < 3; ++d) {
+            const double* src = P + (((size_t)c * 3 + d) * E + e) * kQ3;
+            for (int x = 0; x < NQ; ++x)
+                bulk_load(sX + d * C::kES0 + x * C::kPS0, src + x * NQ * NQ,
+                          (unsigned)(NQ * NQ * sizeof(double)), bar);
+        }
+    };
+
+    long long e = blockIdx.x;
+    if (threadIdx.x == 0 && e < E) fetch(0, e, true);
+    unsigned parity = 0;
+    for (; e < E; e += gridDim.x) {
+        for (int c = 0; c < 3; ++c) {
+            if (!wait_bulk(bar, parity)) return;
+            parity ^= 1u;
+            // stage 1: three products, 3 * kTiles tile tasks dealt round-robin
+            for (int task = warp; task < 3 * S1::kTiles; task += C::kWarps) {
+                const int d = task / S1::kTiles, t = task - d * S1::kTiles;
+                double acc[S1::kMTiles][2];
+#pragma unroll
+                for (int mt = 0; mt < S1::kMTiles; ++mt) acc[mt][0] = acc[mt][1] = 0.0;
+                tile_accumulate<S1, true>(acc, d == 2 ? opD : opI, sX + d * C::kES0, sM, t, lane);
+                tile_store<S1, false>(acc, sT + d * C::kES1, t, lane);
+            }
+            __syncthreads();
+            // the P buffers (and, after the last component, M) are free: fetch what comes next
+            if (threadIdx.x == 0) {
+                const bool last = (c == 2);
+                const long long ne = last ? e + gridDim.x : e;
+                if (ne < E) {
+                    fence_async_proxy();
+                    fetch(last ? 0 : c + 1, ne, last);
+                }
+            }
+            // stage 2: w0 = I t0 (first kTiles tasks), w12 = D t1 + I t2 (the rest)
+            for (int task = warp; task < 2 * S2::kTiles; task += C::kWarps) {
+                const bool dual = task >= S2::kTiles;
+                const int t = dual ? task - S2::kTiles : task;
+                double acc[S2::kMTiles][2];
+#pragma unroll
+                for (int mt = 0; mt < S2::kMTiles; ++mt) acc[mt][0] = acc[mt][1] = 0.0;
+                if (dual) {
+                    tile_accumulate<S2, false>(acc, opD, sT + C::kES1, nullptr, t, lane);
+                    tile_accumulate<S2, false>(acc, opI, sT + 2 * C::kES1, nullptr, t, lane);
+                } else {
+                    tile_accumulate<S2, false>(acc, opI, sT, nullptr, t, lane);
+                }
+                tile_store<S2, false>(acc, sW + (dual ? C::kES2 : 0), t, lane);
+            }
+            __syncthreads();
+            // stage 3: F = D w0 + I w12, straight to global memory in natural order
+            double* Fe = F + ((size_t)c * E + e) * kV3;
+            for (int t = warp; t < S3::kTiles; t += C::kWarps) {
+                double acc[S3::kMTiles][2];
+#pragma unroll
+                for (int mt = 0; mt < S3::kMTiles; ++mt) acc[mt][0] = acc[mt][1] = 0.0;
+                tile_accumulate<S3, false>(acc, opD, sW, nullptr, t, lane);
+                tile_accumulate<S3, false>(acc, opI, sW + C::kES2, nullptr, t, lane);
+                tile_store<S3, true>(acc, Fe, t, lane);
+            }
+            // the next stage 1 writes sT, which stage 2 no longer reads; the next stage 2
+            // writes sW only after the barrier that follows the next stage 1
+        }
+    }
+}
+
+}  // namespace dmma
+}  // namespace ekl

@@ -45,6 +45,9 @@ inline bool apply_fits(int n0, int n1, int n2, int m0, int m1, int m2, size_t el
 // Records the cudaError_t that ekl_tpo_last_cuda_error() reports for the calling thread.
 void set_last_cuda_error(int err);
 
+// Bulk-copy timeout flag of the convective-flux kernels (see ekl_tpo_device_error_flags).
+int convection_timeout_flag();
+
 // Number of SMs of the current device (cached per device).
 int sm_count();
 

@@ -28,8 +28,21 @@
 namespace ekl {
 namespace dmma {
 
-// Set by a kernel whose bounded wait on a bulk copy gave up (not expected in practice).
-__device__ int g_bulk_wait_timeout = 0;
+// Set by a kernel whose bounded wait on a bulk copy gave up (not expected in practice).  Every
+// translation unit that includes this header has its own copy and reads it with
+// take_timeout_flag().
+static __device__ int g_bulk_wait_timeout = 0;
+
+// Host: this translation unit's flag (1 = a wait gave up, -1 = the query failed), cleared.
+static inline int take_timeout_flag() {
+    int flag = 0;
+    if (cudaMemcpyFromSymbol(&flag, g_bulk_wait_timeout, sizeof(int)) != cudaSuccess) return -1;
+    if (flag) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_bulk_wait_timeout, &zero, sizeof(int));
+    }
+    return flag ? 1 : 0;
+}
 
 __device__ __forceinline__ void mma_f64(double& c0, double& c1, double a, double b) {
     asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"

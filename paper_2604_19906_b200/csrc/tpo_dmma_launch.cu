@@ -143,13 +143,8 @@ template bool try_launch_apply_dmma<float>(const float*, const float*, const flo
 // did: bit 0 = a bounded wait on a bulk copy gave up, so the results of that launch are
 // not valid.  Synchronises the device.
 extern "C" int ekl_tpo_device_error_flags(void) {
-    int flag = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-    if (cudaMemcpyFromSymbol(&flag, ekl::dmma::g_bulk_wait_timeout, sizeof(int)) != cudaSuccess)
-        return -1;
-    if (flag) {
-        const int zero = 0;
-        cudaMemcpyToSymbol(ekl::dmma::g_bulk_wait_timeout, &zero, sizeof(int));
-    }
-    return flag ? 1 : 0;
+    const int a = ekl::dmma::take_timeout_flag(), b = ekl::convection_timeout_flag();
+    if (a < 0 || b < 0) return -1;
+    return (a | b) ? 1 : 0;
 }

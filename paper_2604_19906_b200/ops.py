@@ -137,6 +137,34 @@ def ekl_tpo_apply_f32(A, B, C, u, out=None):
     return _apply("ekl_tpo_apply_f32", torch.float32, A, B, C, u, out)
 
 
+def ekl_tpo_convection(Dvq, Ivq, M, P, out=None):
+    """Volume integral of the convective flux: ``F[c,e] = (I⊗I⊗D)(M∘P[c,0]) + (I⊗D⊗I)(M∘P[c,1])
+    + (D⊗I⊗I)(M∘P[c,2])`` in fp64 on the current stream; P is [3,3,E,nq,nq,nq], F [3,E,nv,nv,nv]."""
+    lib = library()
+    fn = lib.ekl_tpo_convection
+    fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
+                                           ctypes.c_void_p]
+    fn.restype = ctypes.c_int
+    if Dvq.dim() != 2 or Dvq.shape != Ivq.shape or M.dim() != 4 or P.dim() != 6:
+        raise ValueError("expected Dvq,Ivq [nv,nq], M [E,nq,nq,nq], P [3,3,E,nq,nq,nq]")
+    nv, nq = Dvq.shape
+    E = M.shape[0]
+    if tuple(M.shape[1:]) != (nq, nq, nq) or tuple(P.shape) != (3, 3, E, nq, nq, nq):
+        raise ValueError("expected M [E,nq,nq,nq] and P [3,3,E,nq,nq,nq]")
+    dev = M.device
+    if out is None:
+        out = torch.empty((3, E, nv, nv, nv), dtype=torch.float64, device=dev)
+    elif tuple(out.shape) != (3, E, nv, nv, nv):
+        raise ValueError("out must be [3,E,nv,nv,nv]")
+    ptrs = [_dev_ptr(t, nm, torch.float64, dev)
+            for t, nm in ((Dvq, "Dvq"), (Ivq, "Ivq"), (M, "M"), (P, "P"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = fn(*ptrs, nq, nv, E, _stream(dev))
+    if st:
+        raise EklTpoError(st, "ekl_tpo_convection")
+    return out
+
+
 def ekl_tpo_version() -> int:
     return int(library().ekl_tpo_version())
 

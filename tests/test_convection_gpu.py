@@ -1,0 +1,75 @@
+"""Convective-flux volume integral (Eq. 1) on the GPU against the oracle."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL64 = 1e-12
+PAIRS = [(4, 4), (6, 4), (6, 6), (8, 4), (8, 6), (8, 8), (10, 8), (10, 10), (12, 8), (12, 10),
+         (12, 12), (14, 12)]
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    import oracle
+    from paper_2604_19906_b200 import build, ops
+    build.build()
+    return {"torch": torch, "oracle": oracle, "ops": ops, "dev": torch.device("cuda:0")}
+
+
+def case(nq, nv, E, seed):
+    g = np.random.Generator(np.random.PCG64(seed))
+    Dvq = g.standard_normal((nv, nq)) / np.sqrt(nq)
+    Ivq = g.standard_normal((nv, nq)) / np.sqrt(nq)
+    M = g.uniform(0.5, 1.5, (E, nq, nq, nq))
+    P = g.uniform(-1, 1, (3, 3, E, nq, nq, nq))
+    return Dvq, Ivq, M, P
+
+
+@pytest.mark.parametrize("nq,nv", PAIRS)
+@pytest.mark.parametrize("E", [1, 2, 5, 311])
+def test_convection_matches_oracle(env, nq, nv, E):
+    torch = env["torch"]
+    Dvq, Ivq, M, P = case(nq, nv, E, 100 * nq + nv + E)
+    want = env["oracle"].convection(Dvq, Ivq, M, P)
+    dev = [torch.from_numpy(np.ascontiguousarray(x)).to(env["dev"]) for x in (Dvq, Ivq, M, P)]
+    got = env["ops"].ekl_tpo_convection(*dev)
+    torch.cuda.synchronize()
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().reshape(3 * E, nv, nv, nv),
+                                            want.reshape(3 * E, nv, nv, nv))
+    assert err.max() <= TOL64, (nq, nv, E, err.max())
+
+
+def test_convection_repeatable_guards_and_errors(env):
+    torch, ops = env["torch"], env["ops"]
+    nq, nv, E = 12, 8, 700
+    Dvq, Ivq, M, P = case(nq, nv, E, 5)
+    dev = [torch.from_numpy(np.ascontiguousarray(x)).to(env["dev"]) for x in (Dvq, Ivq, M, P)]
+    pad = 256
+    big = torch.full((3 * E * nv ** 3 + 2 * pad,), float("nan"), dtype=torch.float64,
+                     device=env["dev"])
+    big[:pad] = 7.0
+    big[-pad:] = 9.0
+    out = big[pad:-pad].view(3, E, nv, nv, nv)
+    ops.ekl_tpo_convection(*dev, out=out)
+    first = out.clone()
+    out.fill_(float("nan"))
+    ops.ekl_tpo_convection(*dev, out=out)
+    assert torch.equal(first, out) and not bool(torch.isnan(out).any())
+    assert bool((big[:pad] == 7.0).all()) and bool((big[-pad:] == 9.0).all())
+    want = env["oracle"].convection(Dvq, Ivq, M, P)
+    err = env["oracle"].rel_err_per_element(out.cpu().numpy().reshape(3 * E, nv, nv, nv),
+                                            want.reshape(3 * E, nv, nv, nv))
+    assert err.max() <= TOL64
+    # unsupported extents and a misaligned field are refused before anything runs
+    D5 = torch.zeros(5, 7, dtype=torch.float64, device=env["dev"])
+    M7 = torch.zeros(2, 7, 7, 7, dtype=torch.float64, device=env["dev"])
+    P7 = torch.zeros(3, 3, 2, 7, 7, 7, dtype=torch.float64, device=env["dev"])
+    with pytest.raises(ops.EklTpoError, match="UNSUPPORTED"):
+        ops.ekl_tpo_convection(D5, D5.clone(), M7, P7)
+    buf = torch.zeros(E * nq ** 3 + 1, dtype=torch.float64, device=env["dev"])
+    with pytest.raises(ops.EklTpoError, match="ALIGN"):
+        ops.ekl_tpo_convection(dev[0], dev[1], buf[1:].view(E, nq, nq, nq), dev[3])
+    lib = ops.library()
+    assert lib.ekl_tpo_device_error_flags() == 0

@@ -21,6 +21,8 @@ from __future__ import annotations
 
 import argparse
 import json
+
+import numpy as np
 import os
 import statistics
 import sys
@@ -125,6 +127,9 @@ def oracle_run(wl, e0, e1):
     t0 = time.perf_counter()
     if wl.op == "inv_helmholtz":
         v = oracle.inv_helmholtz(host["S"], host["D"], host["u"])
+    elif wl.op == "convection":
+        v = oracle.convection(host["Dvq"], host["Ivq"], host["M"], host["P"])
+        v = np.ascontiguousarray(np.moveaxis(v, 0, 1))        # [E,3,nv,nv,nv]: element first
     else:
         v = oracle.tpo_apply(host["A"], host["B"], host["C"], host["u"])
     return time.perf_counter() - t0, v, host
@@ -163,6 +168,8 @@ def reference_arm(args, wl, rank):
     def step():
         if wl.op == "inv_helmholtz":
             oracle.inv_helmholtz(host["S"], host["D"], host["u"])
+        elif wl.op == "convection":
+            oracle.convection(host["Dvq"], host["Ivq"], host["M"], host["P"])
         else:
             oracle.tpo_apply(host["A"], host["B"], host["C"], host["u"])
 
@@ -248,6 +255,14 @@ def main():
         a = (case["S"].data_ptr(), case["D"].data_ptr(), case["u"].data_ptr(), v.data_ptr(),
              wl.n[0], E)
         fn = lib.ekl_tpo_inv_helmholtz
+    elif wl.op == "convection":
+        v = torch.empty((3, E) + tuple(wl.m), dtype=torch.float64, device=dev)
+        a = (case["Dvq"].data_ptr(), case["Ivq"].data_ptr(), case["M"].data_ptr(),
+             case["P"].data_ptr(), v.data_ptr(), wl.n[0], wl.m[0], E)
+        fn = lib.ekl_tpo_convection
+        import ctypes as _ct
+        fn.argtypes = [_ct.c_void_p] * 5 + [_ct.c_int, _ct.c_int, _ct.c_longlong, _ct.c_void_p]
+        fn.restype = _ct.c_int
     else:
         v = torch.empty((E,) + tuple(wl.m), dtype=torch.float64, device=dev)
         a = (case["A"].data_ptr(), case["B"].data_ptr(), case["C"].data_ptr(),
@@ -299,7 +314,8 @@ def main():
     max_rel_err = None
     if base is not None:
         import oracle
-        got = v[:ns_oracle].cpu().numpy()
+        got = (v[:, :ns_oracle].permute(1, 0, 2, 3, 4).contiguous() if wl.op == "convection"
+               else v[:ns_oracle]).cpu().numpy()
         max_rel_err = float(oracle.rel_err_per_element(got, v_oracle).max())
 
     # ---------------------------------------------------------------- FP64 rate of this device, live
@@ -326,7 +342,7 @@ def main():
 
     # ---------------------------------------------------------------- end to end with host buffers
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and wl.op != "convection":
         e2e = run_e2e(torch, ops, wl, case, dev, stream, args.e2e_steps, world, dist)
 
     if rank != 0:

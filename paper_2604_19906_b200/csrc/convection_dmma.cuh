@@ -132,6 +132,17 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
     if (threadIdx.x == 0 && e < E) fetch(0, e, true);
     unsigned parity = 0;
     for (; e < E; e += gridDim.x) {
+        // ask L2 for everything this element still needs and for the first fields of the
+        // next one, a whole element of work ahead of the bulk copies that will use them
+        if (threadIdx.x == 0) {
+            const unsigned field = (unsigned)(kQ3 * sizeof(double));
+            for (int cd = 3; cd < 9; ++cd) bulk_prefetch_l2(P + ((size_t)cd * E + e) * kQ3, field);
+            const long long ne = e + gridDim.x;
+            if (ne < E) {
+                bulk_prefetch_l2(M + (size_t)ne * kQ3, field);
+                for (int d = 0; d < 3; ++d) bulk_prefetch_l2(P + ((size_t)d * E + ne) * kQ3, field);
+            }
+        }
         for (int c = 0; c < 3; ++c) {
             if (!wait_bulk(bar, parity)) return;
             parity ^= 1u;

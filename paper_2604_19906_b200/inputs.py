@@ -42,6 +42,8 @@ _M2 = np.uint64(0x94D049BB133111EB)
 # array ids mixed into the key so that u, c_e, ... are independent streams
 ARRAY_U = 1
 ARRAY_C = 2
+ARRAY_M = 3
+ARRAY_P = 4
 
 
 @dataclass(frozen=True)
@@ -62,18 +64,25 @@ class Workload:
     def name(self) -> str:
         if self.op == "inv_helmholtz":
             return f"cfg{self.index}:inv_helmholtz_{self.dtype}_n{self.n[0]}_E{self.E}"
+        if self.op == "convection":
+            return f"cfg{self.index}:convection_{self.dtype}_nq{self.n[0]}_nv{self.m[0]}_E{self.E}"
         return (f"cfg{self.index}:apply_{self.dtype}_{self.n[0]}x{self.n[1]}x{self.n[2]}"
                 f"_to_{self.m[0]}x{self.m[1]}x{self.m[2]}_E{self.E}")
 
     @property
     def flops_per_element(self) -> int:
-        """Algorithmic flops: 12n⁴+n³ (inverse Helmholtz) or, contraction order
-        C→B→A, 2·(n0·n1·m2·n2 + n0·m1·m2·n1 + m0·m1·m2·n0)."""
+        """Algorithmic flops: 12n⁴+n³ (inverse Helmholtz); contraction order C→B→A,
+        2·(n0·n1·m2·n2 + n0·m1·m2·n1 + m0·m1·m2·n0) (forward operator); for the convective
+        flux nine such forward operators (3 components × 3 directions) plus the 9 nq³
+        products with M and the 6 nv³ additions."""
         n0, n1, n2 = self.n
         m0, m1, m2 = self.m
         if self.op == "inv_helmholtz":
             return 12 * n0 ** 4 + n0 ** 3
-        return 2 * (n0 * n1 * m2 * n2 + n0 * m1 * m2 * n1 + m0 * m1 * m2 * n0)
+        tpo = 2 * (n0 * n1 * m2 * n2 + n0 * m1 * m2 * n1 + m0 * m1 * m2 * n0)
+        if self.op == "convection":
+            return 9 * tpo + 9 * n0 * n1 * n2 + 6 * m0 * m1 * m2
+        return tpo
 
     @property
     def bytes_per_element(self) -> int:
@@ -83,6 +92,8 @@ class Workload:
         nout = self.m[0] * self.m[1] * self.m[2]
         if self.op == "inv_helmholtz":
             return 3 * w * nin
+        if self.op == "convection":
+            return w * (10 * nin + 3 * nout)          # M, nine P fields in; three F fields out
         return w * (nin + nout)
 
 
@@ -92,6 +103,9 @@ CONFIGS = (
     Workload(2, "inv_helmholtz", (12, 12, 12), (12, 12, 12), 65536),
     Workload(3, "inv_helmholtz", (14, 14, 14), (14, 14, 14), 131072),
     Workload(4, "apply", (8, 8, 8), (12, 12, 12), 131072),
+    # not one of the five stated configurations: the convective-flux integral of Eq. 1 on the
+    # paper's batch size (8192 elements per call), 12 quadrature -> 8 volume points
+    Workload(5, "convection", (12, 12, 12), (8, 8, 8), 8192),
 )
 
 
@@ -168,9 +182,34 @@ def host_D(wl: Workload, lam: np.ndarray, e0: int, e1: int) -> np.ndarray:
     return 1.0 / (s[None, :, :, :] + c[:, None, None, None])
 
 
+def host_M(wl: Workload, e0: int, e1: int) -> np.ndarray:
+    """M[e0:e1] ~ U(0.5,1.5), shape [e1-e0, nq, nq, nq]."""
+    per = wl.n[0] * wl.n[1] * wl.n[2]
+    x = counter_uniform(stream_key(wl.seed, ARRAY_M), e0 * per, (e1 - e0) * per, 0.5, 1.5)
+    return x.reshape((e1 - e0,) + tuple(wl.n))
+
+
+def host_P(wl: Workload, e0: int, e1: int) -> np.ndarray:
+    """P[:, :, e0:e1] ~ U(-1,1), shape [3,3,e1-e0,nq,nq,nq]; the stream index is that of the
+    full [3,3,E,...] array."""
+    per = wl.n[0] * wl.n[1] * wl.n[2]
+    key = stream_key(wl.seed, ARRAY_P)
+    out = np.empty((3, 3, e1 - e0) + tuple(wl.n))
+    for c in range(3):
+        for d in range(3):
+            start = ((c * 3 + d) * wl.E + e0) * per
+            out[c, d] = counter_uniform(key, start, (e1 - e0) * per, -1.0, 1.0).reshape(
+                (e1 - e0,) + tuple(wl.n))
+    return out
+
+
 def host_case(wl: Workload, e0: int = 0, e1: int | None = None) -> dict:
     """All inputs of ``wl`` for elements [e0,e1) as NumPy arrays (fp64)."""
     e1 = wl.E if e1 is None else e1
+    if wl.op == "convection":
+        return {"Dvq": gaussian_factor(wl.m[0], wl.n[0], wl.seed, 0),
+                "Ivq": gaussian_factor(wl.m[0], wl.n[0], wl.seed, 1),
+                "M": host_M(wl, e0, e1), "P": host_P(wl, e0, e1)}
     if wl.op == "inv_helmholtz":
         n = wl.n[0]
         lam = eigen_lambda(n, wl.seed)
@@ -215,6 +254,26 @@ def device_case(wl: Workload, device="cuda:0", e0: int = 0, e1: int | None = Non
     lib = _fill_lib()
     per = wl.n[0] * wl.n[1] * wl.n[2]
     out = {}
+    if wl.op == "convection":
+        with torch.cuda.device(dev):
+            st = torch.cuda.current_stream(dev).cuda_stream
+            M = torch.empty((E,) + tuple(wl.n), dtype=torch.float64, device=dev)
+            P = torch.empty((3, 3, E) + tuple(wl.n), dtype=torch.float64, device=dev)
+            rc = lib.ekl_inputs_fill_uniform_f64(M.data_ptr(), e0 * per, E * per,
+                                                 stream_key(wl.seed, ARRAY_M), 0.5, 1.0, st) if E else 0
+            for c in range(3):
+                for d in range(3):
+                    if E and not rc:
+                        rc = lib.ekl_inputs_fill_uniform_f64(
+                            P[c, d].data_ptr(), ((c * 3 + d) * wl.E + e0) * per, E * per,
+                            stream_key(wl.seed, ARRAY_P), -1.0, 2.0, st)
+            if rc:
+                raise RuntimeError(f"fill_uniform failed with CUDA error {rc}")
+            out = {"M": M, "P": P,
+                   "Dvq": torch.from_numpy(gaussian_factor(wl.m[0], wl.n[0], wl.seed, 0)).to(dev),
+                   "Ivq": torch.from_numpy(gaussian_factor(wl.m[0], wl.n[0], wl.seed, 1)).to(dev)}
+            torch.cuda.synchronize(dev)
+        return out
     with torch.cuda.device(dev):
         st = torch.cuda.current_stream(dev).cuda_stream
         u = torch.empty((E,) + tuple(wl.n), dtype=torch.float64, device=dev)

@@ -73,3 +73,22 @@ def test_convection_repeatable_guards_and_errors(env):
         ops.ekl_tpo_convection(dev[0], dev[1], buf[1:].view(E, nq, nq, nq), dev[3])
     lib = ops.library()
     assert lib.ekl_tpo_device_error_flags() == 0
+
+
+def test_convection_workload_full_size_sampled(env):
+    """The benchmark's convection workload (nq = 12, nv = 8, E = 8192) generated on the
+    device, every element computed, the oracle recomputing runs at both ends and the middle."""
+    torch = env["torch"]
+    from paper_2604_19906_b200 import inputs
+    wl = inputs.CONFIGS[5]
+    case_d = inputs.device_case(wl, env["dev"])
+    got = env["ops"].ekl_tpo_convection(case_d["Dvq"], case_d["Ivq"], case_d["M"], case_d["P"])
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(got).all())
+    E, nv = wl.E, wl.m[0]
+    for e0, e1 in ((0, 64), (E // 2 - 30, E // 2 + 41), (E - 50, E)):
+        h = inputs.host_case(wl, e0, e1)
+        want = env["oracle"].convection(h["Dvq"], h["Ivq"], h["M"], h["P"])
+        g = got[:, e0:e1].cpu().numpy()
+        err = env["oracle"].rel_err_per_element(g.reshape(-1, nv, nv, nv), want.reshape(-1, nv, nv, nv))
+        assert err.max() <= TOL64, (e0, err.max())

@@ -288,7 +288,7 @@ def test_runtime_argument_errors_raise(env):
 
 def test_device_input_generators_match_the_host_bit_for_bit(env):
     inputs = env["inputs"]
-    for idx in (0, 1, 4):
+    for idx in (0, 1, 4, 5):
         wl = inputs.CONFIGS[idx]
         e0, e1 = 5, min(wl.E, 45)
         host = inputs.host_case(wl, e0, e1)

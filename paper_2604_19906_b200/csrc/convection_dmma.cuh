@@ -147,7 +147,10 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             if (!wait_bulk(bar, parity)) return;
             parity ^= 1u;
             // stage 1: three products, 3 * kTiles tile tasks dealt round-robin
-            for (int task = warp; task < 3 * S1::kTiles; task += C::kWarps) {
+#pragma unroll
+            for (int it = 0; it < (3 * S1::kTiles + C::kWarps - 1) / C::kWarps; ++it) {
+                const int task = warp + it * C::kWarps;
+                if (task >= 3 * S1::kTiles) break;
                 const int d = task / S1::kTiles, t = task - d * S1::kTiles;
                 double acc[S1::kMTiles][2];
 #pragma unroll
@@ -166,7 +169,10 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
                 }
             }
             // stage 2: w0 = I t0 (first kTiles tasks), w12 = D t1 + I t2 (the rest)
-            for (int task = warp; task < 2 * S2::kTiles; task += C::kWarps) {
+#pragma unroll
+            for (int it = 0; it < (2 * S2::kTiles + C::kWarps - 1) / C::kWarps; ++it) {
+                const int task = warp + it * C::kWarps;
+                if (task >= 2 * S2::kTiles) break;
                 const bool dual = task >= S2::kTiles;
                 const int t = dual ? task - S2::kTiles : task;
                 double acc[S2::kMTiles][2];
@@ -183,7 +189,10 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             __syncthreads();
             // stage 3: F = D w0 + I w12, straight to global memory in natural order
             double* Fe = F + ((size_t)c * E + e) * kV3;
-            for (int t = warp; t < S3::kTiles; t += C::kWarps) {
+#pragma unroll
+            for (int it = 0; it < (S3::kTiles + C::kWarps - 1) / C::kWarps; ++it) {
+                const int t = warp + it * C::kWarps;
+                if (t >= S3::kTiles) break;
                 double acc[S3::kMTiles][2];
 #pragma unroll
                 for (int mt = 0; mt < S3::kMTiles; ++mt) acc[mt][0] = acc[mt][1] = 0.0;

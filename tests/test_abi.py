@@ -90,6 +90,53 @@ def test_apply_validation(lib, fn, w):
     assert f(A, B, C, u, A, *dims, E, None) == OVERLAP
 
 
+def test_convection_and_host_variants_validation(lib):
+    OK, NULL, SHAPE, UNSUP, ALIGN, OVERLAP = 0, 1, 2, 3, 4, 5
+    vp, i, ll, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_size_t
+    f = lib.ekl_tpo_convection
+    f.argtypes = [vp] * 5 + [i, i, ll, vp]
+    f.restype = i
+    nq, nv, E = 12, 8, 4
+    D, I = P, P + 0x1000
+    M = P + 0x2000
+    Pf = M + E * nq ** 3 * 8
+    F = Pf + 0x40000000
+    assert f(D, I, M, Pf, F, nq, nv, 0, None) == OK
+    assert f(D, I, M, Pf, F, 0, nv, E, None) == SHAPE
+    assert f(D, I, M, Pf, F, nq, nv, -1, None) == SHAPE
+    assert f(D, None, M, Pf, F, nq, nv, E, None) == NULL
+    assert f(D, I, M, Pf, F, 13, 8, E, None) == UNSUP            # no instance for these extents
+    assert f(D, I, M, Pf, F, 100, 8, E, None) == UNSUP
+    assert f(D, I, M + 8, Pf, F, nq, nv, E, None) == ALIGN       # M and P need 16 bytes
+    assert f(D, I, M, Pf, F + 4, nq, nv, E, None) == ALIGN
+    assert f(D, I, M, Pf, Pf, nq, nv, E, None) == OVERLAP
+    assert f(D, I, M, Pf, M, nq, nv, E, None) == OVERLAP
+    g = lib.ekl_tpo_inv_helmholtz_host
+    g.argtypes = [vp, vp, vp, vp, i, ll, vp, sz, vp]
+    g.restype = i
+    n = 4
+    S, Dh, u, v = P, P + 0x1000, P + 0x2000, P + 0x3000
+    ws = 0x7F1000000000
+    assert g(S, Dh, u, v, n, 0, None, 0, None) == OK
+    assert g(S, Dh, u, v, 0, 3, ws, 1 << 20, None) == SHAPE
+    assert g(S, Dh, u, v, n, 3, None, 1 << 20, None) == NULL
+    assert g(S, Dh, u, v, 99, 3, ws, 1 << 20, None) == UNSUP
+    assert g(S, Dh, u + 1, v, n, 3, ws, 1 << 20, None) == ALIGN
+    assert g(S, Dh, u, Dh, n, 3, ws, 1 << 20, None) == OVERLAP
+    assert g(S, Dh, u, v, n, 3, ws + 8, 1 << 20, None) == ALIGN   # workspace must be 256-byte aligned
+    assert g(S, Dh, u, v, n, 3, ws, 64, None) == UNSUP            # workspace too small
+    h = lib.ekl_tpo_inv_helmholtz_host_static
+    h.argtypes = [vp, vp, vp, vp, i, ll, vp]
+    h.restype = i
+    assert h(S, Dh, u, v, n, 0, None) == OK
+    assert h(S, Dh, u, v, 14, 510, None) == UNSUP                 # beyond the fixed staging area
+    assert h(S, Dh, None, v, n, 3, None) == NULL
+    w = lib.ekl_tpo_host_workspace_bytes
+    w.argtypes = [ll, i, ll, ll, ll, i]
+    w.restype = sz
+    assert w(64, 2, 64, 16, 10, 8) >= 3 * 10 * 3 * 64 * 8 and w(64, 2, 64, 16, 0, 8) == 0
+
+
 def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     from paper_2604_19906_b200 import ops
     monkeypatch.setattr(ops, "_lib", None)

@@ -181,6 +181,23 @@ def test_inv_helmholtz_many_batches_per_cta(env, n, E):
     assert err.max() <= TOL64, (n, E, err.max())
 
 
+@pytest.mark.parametrize("n,E", [(14, 3001), (12, 2000), (9, 1500), (8, 5000)])
+def test_inv_helmholtz_in_place_with_many_batches_per_cta(env, n, E):
+    """v == u while every persistent CTA streams several batches: a batch's u must be on chip
+    before its v is written, and no CTA may touch another one's elements."""
+    torch = env["torch"]
+    S, D, u = synth_ih(n, E, 9100 + n)
+    Sd, Dd, ud = to_dev(env, S), to_dev(env, D), to_dev(env, u)
+    ref = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud)
+    inplace = ud.clone()
+    env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, inplace, out=inplace)
+    torch.cuda.synchronize()
+    assert torch.equal(inplace, ref)
+    sample = slice(E - 40, E)
+    want = env["oracle"].inv_helmholtz(S, D[sample], u[sample])
+    assert env["oracle"].rel_err_per_element(ref[sample].cpu().numpy(), want).max() <= TOL64
+
+
 def test_no_device_error_flags_after_all_this(env):
     lib = env["ops"].library()
     lib.ekl_tpo_device_error_flags.restype = __import__("ctypes").c_int

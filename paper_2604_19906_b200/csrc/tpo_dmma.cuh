@@ -226,7 +226,12 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
             in + eb * SS::IN_ES + pb1 * SS::IN_RS + (pb - pb1 * SS::E2) + kk * SS::IN_PS;
         double b[SS::kKSteps];
 #pragma unroll
-        for (int s = 0; s < SS::kKSteps; ++s) b[s] = src[SS::k0(s) * SS::IN_PS];
+        for (int s = 0; s < SS::kKSteps; ++s) {
+            // lanes whose contraction index an overlapping last step repeats need no data:
+            // their operator entries are zero
+            const int repeated = (s > 0) ? SS::k0(s - 1) + 4 - SS::k0(s) : 0;
+            b[s] = (kk >= repeated) ? src[SS::k0(s) * SS::IN_PS] : 0.0;
+        }
         double dn[SS::kMTiles][2];
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp)
             load_factor<SS, T>(dn, Db, valid_pencils, warp, slot + 1, lane);

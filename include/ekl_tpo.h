@@ -64,9 +64,9 @@ typedef enum {
  *
  * fp64.  `v == u` exactly (in place) is allowed; any other overlap of v with an
  * input is rejected.  1 <= n; n is limited by shared memory (n <= 24 for fp64).
- * Even n from 4 to 16 with a 16-byte aligned u run on the FP64 tensor path (fastest);
- * every other accepted case runs on a slower general kernel with the same results to
- * rounding.
+ * Every n from 4 to 16 runs on the FP64 tensor path (for even n this needs a 16-byte
+ * aligned u); every other accepted case runs on a slower general kernel with the same
+ * results to rounding.
  */
 ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const double* u,
                                      double* v, int n, long long E, cudaStream_t stream);
@@ -78,7 +78,9 @@ ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const dou
  *
  *   A [m0,n0]  B [m1,n1]  C [m2,n2]     u [E,n0,n1,n2]     v [E,m0,m1,m2]
  *
- * fp64.  v must not overlap any input.
+ * fp64.  v must not overlap any input.  Cubic shapes n -> m (n0=n1=n2, m0=m1=m2) with even
+ * n, m from 4 to 16 and a 16-byte aligned u run on the FP64 tensor path; every other shape
+ * that fits in shared memory runs on the general kernel.
  */
 ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
                              const double* u, double* v,
@@ -108,7 +110,12 @@ ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const do
                                   const double* P, double* F, int nq, int nv, long long E,
                                   cudaStream_t stream);
 
-/* Single-precision twins of the two operators above (same layout and rules). */
+/*
+ * Single-precision twins of ekl_tpo_inv_helmholtz and ekl_tpo_apply (same layout and
+ * rules; tolerance 1e-5 instead of 1e-12).  On the tensor path the fields are widened to
+ * fp64 on chip, all arithmetic is fp64, and v is rounded to fp32 once when it is stored;
+ * the general kernel computes in fp32.
+ */
 ekl_tpo_status ekl_tpo_inv_helmholtz_f32(const float* S, const float* D, const float* u,
                                          float* v, int n, long long E, cudaStream_t stream);
 ekl_tpo_status ekl_tpo_apply_f32(const float* A, const float* B, const float* C,

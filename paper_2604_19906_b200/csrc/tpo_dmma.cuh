@@ -315,6 +315,28 @@ __device__ __forceinline__ void copy_elements(double* dst, const T* __restrict__
     asm volatile("cp.async.commit_group;" ::: "memory");
 }
 
+// All threads: `count` floats from global memory into a dense staging area, asynchronously.
+__device__ __forceinline__ void stage_floats(float* dst, const float* __restrict__ src, int count) {
+    for (int idx = threadIdx.x; idx < count; idx += blockDim.x)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_addr(dst + idx)),
+                     "l"(src + idx)
+                     : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// All threads: widen staged fields (dense, element after element) into the stage-input layout.
+template <int K, int P, int PS, int ES>
+__device__ __forceinline__ void widen_elements(double* dst, const float* src, int cnt) {
+    const int total = cnt * K * P;
+#pragma unroll 4
+    for (int idx = threadIdx.x; idx < total; idx += blockDim.x) {
+        const int e = idx / (K * P);
+        const int rem = idx - e * (K * P);
+        const int x = rem / P;
+        dst[e * ES + x * PS + (rem - x * P)] = (double)src[idx];
+    }
+}
+
 __device__ __forceinline__ void wait_copies() {
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
@@ -322,7 +344,7 @@ __device__ __forceinline__ void wait_copies() {
 
 // ------------------------------------------------------------------ inverse Helmholtz
 
-template <int N>
+template <int N, typename T = double>
 struct IhCfg {
     // natural-order input planes, padded so that the first stage loads without conflicts
     static constexpr int kPS0 = pad_plane(N * N), kES0 = N * kPS0;
@@ -344,7 +366,12 @@ struct IhCfg {
     using Last = Stage<N, N, N, N, kBe, kWarps, kRS, kPS, kES, N, N * N, N * N * N>;
     static constexpr int kThreads = 32 * kWarps;
     static constexpr int kBufElems = kBe * kElemBuf;
-    static constexpr size_t kSmemBytes = 2 * (size_t)kBufElems * sizeof(double) + 16;
+    // single-precision fields land asynchronously in a dense staging area of their own and are
+    // widened into the stage-1 input at the start of their batch
+    static constexpr size_t kStagingBytes =
+        sizeof(T) == sizeof(float) ? ((size_t)kBe * N * N * N * sizeof(float) + 15) / 16 * 16 : 0;
+    static constexpr size_t kSmemBytes =
+        2 * (size_t)kBufElems * sizeof(double) + kStagingBytes + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
     static constexpr int kByWarps = 20 / kWarps;
     static constexpr int kCtasPerSm =
@@ -357,10 +384,10 @@ struct IhCfg {
 // v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])).  T is the type of the fields in memory
 // (double: even N needs 16-byte aligned u; float: widened on load, rounded once on store).
 template <int N, typename T>
-__global__ void __launch_bounds__(IhCfg<N>::kThreads, IhCfg<N>::kCtasPerSm)
+__global__ void __launch_bounds__(IhCfg<N, T>::kThreads, IhCfg<N, T>::kCtasPerSm)
 inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u, T* v,
                    long long E) {
-    using C = IhCfg<N>;
+    using C = IhCfg<N, T>;
     constexpr bool kBulk = C::kBulk && sizeof(T) == sizeof(double);
     using First = typename C::First;
     using Mid = typename C::Mid;
@@ -369,7 +396,10 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
     extern __shared__ __align__(128) unsigned char smem_raw[];
     double* bufA = reinterpret_cast<double*>(smem_raw);
     double* bufB = bufA + C::kBufElems;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(bufB + C::kBufElems);
+    float* staging = reinterpret_cast<float*>(bufB + C::kBufElems);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(staging) +
+                                                C::kStagingBytes);
+    constexpr bool kStaged = sizeof(T) == sizeof(float);
 
     // which warp takes the odd tile out rotates with the CTA, so that co-resident CTAs do
     // not load the same scheduler partition
@@ -391,7 +421,10 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
     };
     long long batch = blockIdx.x;
     if (batch < n_batches) {
-        if (!kBulk)
+        if (kStaged)
+            stage_floats(staging, reinterpret_cast<const float*>(u) + batch * C::kBe * kN3,
+                         batch_count(batch) * kN3);
+        else if (!kBulk)
             copy_elements<N, kN2, C::kPS0, C::kES0, T>(bufA, u + batch * C::kBe * kN3,
                                                     batch_count(batch));
         else if (threadIdx.x == 0)
@@ -417,6 +450,10 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
             parity ^= 1u;
         } else {
             wait_copies();
+            if (kStaged) {
+                widen_elements<N, kN2, C::kPS0, C::kES0>(bufA, staging, cnt);
+                __syncthreads();
+            }
         }
         // forward: contract i, j, k
         run_stage<First, 0, T>(bufA, bufB, nullptr, op, dfac, nullptr, valid, warp, lane);
@@ -434,7 +471,10 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (next < n_batches) {
-            if (!kBulk) {
+            if (kStaged) {
+                stage_floats(staging, reinterpret_cast<const float*>(u) + next * C::kBe * kN3,
+                             batch_count(next) * kN3);
+            } else if (!kBulk) {
                 copy_elements<N, kN2, C::kPS0, C::kES0, T>(bufA, u + next * C::kBe * kN3,
                                                         batch_count(next));
             } else if (threadIdx.x == 0) {

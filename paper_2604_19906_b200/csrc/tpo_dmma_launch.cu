@@ -32,7 +32,7 @@ cudaError_t ctas_per_sm(Kernel kernel, int threads, size_t smem, int (&cached)[6
 
 template <int N, typename T>
 cudaError_t launch_ih(const T* S, const T* D, const T* u, T* v, long long E, cudaStream_t stream) {
-    using C = dmma::IhCfg<N>;
+    using C = dmma::IhCfg<N, T>;
     static int cached[64] = {0};
     int per_sm = 1;
     cudaError_t err =

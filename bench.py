@@ -233,16 +233,22 @@ def main():
 
     import torch
     from paper_2604_19906_b200 import build, ops, sharding
-    build.build()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if local_rank >= torch.cuda.device_count():
+        raise SystemExit(f"LOCAL_RANK {local_rank} but only {torch.cuda.device_count()} GPU(s) visible")
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+        # one process per node (re)builds the in-tree libraries, the others wait for it
+        if local_rank == 0:
+            build.build()
+        dist.barrier()
     else:
         dist = None
+        build.build()
     if world != args.gpus and rank == 0:
         print(f"# note: --gpus {args.gpus} but WORLD_SIZE={world}", file=sys.stderr)
 

@@ -355,7 +355,7 @@ struct IhCfg {
     static constexpr int kBe = (N <= 6) ? 4 : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
     static constexpr int kWarps = (N == 14)           ? 8
-                                  : (kTiles <= 16 && kTiles % 4 == 0) ? 4
+                                  : (kTiles <= 36 && kTiles % 4 == 0) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6
                                   : (kTiles % 5 == 0) ? 5

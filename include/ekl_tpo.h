@@ -101,10 +101,11 @@ ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
  *
  * i.e. F[c,e,k,j,i] = sum_{l,m,n} ( D[i,l] I[j,m] I[k,n] P[c,0,e,n,m,l] + I[i,l] D[j,m] I[k,n]
  * P[c,1,e,n,m,l] + I[i,l] I[j,m] D[k,n] P[c,2,e,n,m,l] ) M[e,n,m,l]: the derivative acts on the
- * fastest axis for direction 0 and on the slowest for direction 2.  fp64.  M and P must be
- * 16-byte aligned (EKL_TPO_ERR_ALIGN otherwise); F must not overlap any input.  Available
- * for (nq,nv) in {(4,4),(6,4),(6,6),(8,4),(8,6),(8,8),(10,8),(10,10),(12,8),(12,10),(12,12),
- * (14,12)}; other extents return EKL_TPO_ERR_UNSUPPORTED.
+ * fastest axis for direction 0 and on the slowest for direction 2.  fp64.  F must not
+ * overlap any input.  (nq,nv) in {(4,4),(6,4),(6,6),(8,4),(8,6),(8,8),(10,8),(10,10),(12,8),
+ * (12,10),(12,12),(14,12)} with 16-byte aligned M and P run on the FP64 tensor path; every
+ * other combination that fits in shared memory (nq, nv <= 64 and about 2 max(nq,nv)^3 + nv^3
+ * values) runs on a general kernel; larger extents return EKL_TPO_ERR_UNSUPPORTED.
  */
 ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const double* M,
                                   const double* P, double* F, int nq, int nv, long long E,

@@ -50,10 +50,13 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
     if (nq < 1 || nv < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
     if (E == 0) return EKL_TPO_OK;
     if (!Dvq || !Ivq || !M || !P || !F) return EKL_TPO_ERR_NULL;
-    if (nq > 64 || nv > 64) return EKL_TPO_ERR_UNSUPPORTED;
-    if (misaligned(Dvq, 8) || misaligned(Ivq, 8) || misaligned(F, 8) || misaligned(M, 16) ||
-        misaligned(P, 16))
+    if (nq > 64 || nv > 64 || ekl::generic_conv_smem(nq, nv) > ekl::kMaxSmemBytes)
+        return EKL_TPO_ERR_UNSUPPORTED;
+    if (misaligned(Dvq, 8) || misaligned(Ivq, 8) || misaligned(F, 8) || misaligned(M, 8) ||
+        misaligned(P, 8))
         return EKL_TPO_ERR_ALIGN;
+    // the tensor-path instances bulk-copy M and P: 16-byte aligned fields
+    const bool tensor_ok = ekl::tuned_kernels_allowed() && !misaligned(M, 16) && !misaligned(P, 16);
     const size_t q3 = (size_t)nq * nq * nq * sizeof(double), v3 = (size_t)nv * nv * nv * sizeof(double);
     const size_t fbytes = 3 * (size_t)E * v3, mat = (size_t)nv * nq * sizeof(double);
     if (overlaps(F, fbytes, M, (size_t)E * q3) || overlaps(F, fbytes, P, 9 * (size_t)E * q3) ||
@@ -61,7 +64,7 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
         return EKL_TPO_ERR_OVERLAP;
     cudaError_t err = cudaSuccess;
 #define EKL_CONV_CASE(Q, V)                                                   \
-    if (nq == Q && nv == V) {                                                 \
+    if (tensor_ok && nq == Q && nv == V) {                                    \
         err = launch_conv<Q, V>(Dvq, Ivq, M, P, F, E, stream);                \
         if (err != cudaSuccess) {                                             \
             ekl::set_last_cuda_error((int)err);                               \
@@ -82,5 +85,10 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
     EKL_CONV_CASE(12, 12)
     EKL_CONV_CASE(14, 12)
 #undef EKL_CONV_CASE
-    return EKL_TPO_ERR_UNSUPPORTED;
+    err = ekl::launch_convection_generic(Dvq, Ivq, M, P, F, nq, nv, E, stream);
+    if (err != cudaSuccess) {
+        ekl::set_last_cuda_error((int)err);
+        return EKL_TPO_ERR_CUDA;
+    }
+    return EKL_TPO_OK;
 }

@@ -45,8 +45,28 @@ inline bool apply_fits(int n0, int n1, int n2, int m0, int m1, int m2, size_t el
 // Records the cudaError_t that ekl_tpo_last_cuda_error() reports for the calling thread.
 void set_last_cuda_error(int err);
 
+// Run-time-sized convective-flux kernel: elements of one ping-pong buffer, total shared
+// memory, launcher.
+inline size_t generic_conv_buf(int nq, int nv) {
+    size_t a = (size_t)nq * nq * nq, b = (size_t)nq * nq * nv, c = (size_t)nq * nv * nv,
+           d = (size_t)nv * nv * nv;
+    size_t m = a > b ? a : b;
+    m = m > c ? m : c;
+    return m > d ? m : d;
+}
+inline size_t generic_conv_smem(int nq, int nv) {
+    return (2 * (size_t)nv * nq + 2 * generic_conv_buf(nq, nv) + (size_t)nv * nv * nv) *
+           sizeof(double);
+}
+cudaError_t launch_convection_generic(const double* Dvq, const double* Ivq, const double* M,
+                                      const double* P, double* F, int nq, int nv, long long E,
+                                      cudaStream_t stream);
+
 // Bulk-copy timeout flag of the convective-flux kernels (see ekl_tpo_device_error_flags).
 int convection_timeout_flag();
+
+// False when EKL_TPO_VARIANT=generic asks for the run-time-sized kernels only.
+bool tuned_kernels_allowed();
 
 // Number of SMs of the current device (cached per device).
 int sm_count();

@@ -92,4 +92,46 @@ __global__ void apply_generic(const T* __restrict__ A, const T* __restrict__ B,
     }
 }
 
+// F[c,e] = (I(x)I(x)D)(M[e] o P[c,0,e]) + (I(x)D(x)I)(M[e] o P[c,1,e]) + (D(x)I(x)I)(M[e] o P[c,2,e])
+// for run-time extents: one CTA per (component, element) pair at a time, the three forward
+// operators evaluated one after the other and summed in a shared accumulator.
+template <typename T>
+__global__ void convection_generic(const T* __restrict__ Dvq, const T* __restrict__ Ivq,
+                                   const T* __restrict__ M, const T* __restrict__ P,
+                                   T* __restrict__ F, int nq, int nv, int buf_elems, long long E) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T* sD = reinterpret_cast<T*>(smem_raw);
+    T* sI = sD + nv * nq;
+    T* b0 = sI + nv * nq;
+    T* b1 = b0 + buf_elems;
+    T* acc = b1 + buf_elems;
+    for (int x = threadIdx.x; x < nv * nq; x += blockDim.x) {
+        sD[x] = Dvq[x];
+        sI[x] = Ivq[x];
+    }
+    const int q3 = nq * nq * nq, v3 = nv * nv * nv;
+    for (long long w = blockIdx.x; w < 3 * E; w += gridDim.x) {
+        const long long c = w / E, e = w - c * E;
+        const T* Me = M + e * q3;
+        for (int d = 0; d < 3; ++d) {
+            const T* Pd = P + ((c * 3 + d) * E + e) * q3;
+            __syncthreads();  // b0, b1 and acc of the previous pass are no longer read
+            for (int x = threadIdx.x; x < q3; x += blockDim.x) b0[x] = Me[x] * Pd[x];
+            __syncthreads();
+            // the derivative matrix sits on the fastest axis for d = 0, the slowest for d = 2
+            contract_axis<T, T>(b0, b1, d == 0 ? sD : sI, nq, 1, nq, nq, nq, 2, nv, nullptr);
+            __syncthreads();
+            contract_axis<T, T>(b1, b0, d == 1 ? sD : sI, nq, 1, nq, nq, nv, 1, nv, nullptr);
+            __syncthreads();
+            contract_axis<T, T>(b0, b1, d == 2 ? sD : sI, nq, 1, nq, nv, nv, 0, nv, nullptr);
+            __syncthreads();
+            for (int x = threadIdx.x; x < v3; x += blockDim.x)
+                acc[x] = (d == 0) ? b1[x] : acc[x] + b1[x];
+        }
+        __syncthreads();
+        T* Fe = F + (c * E + e) * v3;
+        for (int x = threadIdx.x; x < v3; x += blockDim.x) Fe[x] = acc[x];
+    }
+}
+
 }  // namespace ekl

@@ -79,6 +79,28 @@ static bool tuned_allowed() {
     return allowed;
 }
 
+cudaError_t launch_convection_generic(const double* Dvq, const double* Ivq, const double* M,
+                                      const double* P, double* F, int nq, int nv, long long E,
+                                      cudaStream_t stream) {
+    const size_t smem = generic_conv_smem(nq, nv);
+    cudaError_t err = cudaFuncSetAttribute(convection_generic<double>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    const int threads = round_up_warp((long long)nq * nq * nv, 512);
+    int per_sm = 1;
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, convection_generic<double>,
+                                                        threads, smem);
+    if (err != cudaSuccess) return err;
+    if (per_sm < 1) per_sm = 1;
+    long long grid = (long long)sm_count() * per_sm;
+    if (grid > 3 * E) grid = 3 * E;
+    convection_generic<double><<<(unsigned)grid, threads, smem, stream>>>(
+        Dvq, Ivq, M, P, F, nq, nv, (int)generic_conv_buf(nq, nv), E);
+    return cudaGetLastError();
+}
+
+bool tuned_kernels_allowed() { return tuned_allowed(); }
+
 template <typename T>
 cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
                                  cudaStream_t stream) {

@@ -105,9 +105,9 @@ def test_convection_and_host_variants_validation(lib):
     assert f(D, I, M, Pf, F, 0, nv, E, None) == SHAPE
     assert f(D, I, M, Pf, F, nq, nv, -1, None) == SHAPE
     assert f(D, None, M, Pf, F, nq, nv, E, None) == NULL
-    assert f(D, I, M, Pf, F, 13, 8, E, None) == UNSUP            # no instance for these extents
-    assert f(D, I, M, Pf, F, 100, 8, E, None) == UNSUP
-    assert f(D, I, M + 8, Pf, F, nq, nv, E, None) == ALIGN       # M and P need 16 bytes
+    assert f(D, I, M, Pf, F, 100, 8, E, None) == UNSUP           # beyond 64
+    assert f(D, I, M, Pf, F, 40, 40, E, None) == UNSUP           # does not fit in shared memory
+    assert f(D, I, M + 4, Pf, F, nq, nv, E, None) == ALIGN
     assert f(D, I, M, Pf, F + 4, nq, nv, E, None) == ALIGN
     assert f(D, I, M, Pf, Pf, nq, nv, E, None) == OVERLAP
     assert f(D, I, M, Pf, M, nq, nv, E, None) == OVERLAP

@@ -62,17 +62,37 @@ def test_convection_repeatable_guards_and_errors(env):
     err = env["oracle"].rel_err_per_element(out.cpu().numpy().reshape(3 * E, nv, nv, nv),
                                             want.reshape(3 * E, nv, nv, nv))
     assert err.max() <= TOL64
-    # unsupported extents and a misaligned field are refused before anything runs
-    D5 = torch.zeros(5, 7, dtype=torch.float64, device=env["dev"])
-    M7 = torch.zeros(2, 7, 7, 7, dtype=torch.float64, device=env["dev"])
-    P7 = torch.zeros(3, 3, 2, 7, 7, 7, dtype=torch.float64, device=env["dev"])
+    # extents beyond shared memory are refused before anything runs
+    D5 = torch.zeros(40, 40, dtype=torch.float64, device=env["dev"])
+    M7 = torch.zeros(1, 40, 40, 40, dtype=torch.float64, device=env["dev"])
+    P7 = torch.zeros(3, 3, 1, 40, 40, 40, dtype=torch.float64, device=env["dev"])
     with pytest.raises(ops.EklTpoError, match="UNSUPPORTED"):
         ops.ekl_tpo_convection(D5, D5.clone(), M7, P7)
+    # M only 8-byte aligned: the general kernel takes over, same result
     buf = torch.zeros(E * nq ** 3 + 1, dtype=torch.float64, device=env["dev"])
-    with pytest.raises(ops.EklTpoError, match="ALIGN"):
-        ops.ekl_tpo_convection(dev[0], dev[1], buf[1:].view(E, nq, nq, nq), dev[3])
+    M8 = buf[1:].view(E, nq, nq, nq)
+    M8.copy_(dev[2])
+    got8 = ops.ekl_tpo_convection(dev[0], dev[1], M8, dev[3])
+    err = env["oracle"].rel_err_per_element(got8.cpu().numpy().reshape(3 * E, nv, nv, nv),
+                                            want.reshape(3 * E, nv, nv, nv))
+    assert err.max() <= TOL64
     lib = ops.library()
     assert lib.ekl_tpo_device_error_flags() == 0
+
+
+@pytest.mark.parametrize("nq,nv", [(3, 2), (5, 7), (7, 5), (9, 9), (13, 8), (16, 12), (2, 1), (1, 1)])
+@pytest.mark.parametrize("E", [1, 4, 97])
+def test_convection_general_kernel_shapes(env, nq, nv, E):
+    """Extents without a tensor-path instance run on the run-time-sized kernel."""
+    torch = env["torch"]
+    Dvq, Ivq, M, P = case(nq, nv, E, 7 * nq + nv + E)
+    want = env["oracle"].convection(Dvq, Ivq, M, P)
+    dev = [torch.from_numpy(np.ascontiguousarray(x)).to(env["dev"]) for x in (Dvq, Ivq, M, P)]
+    got = env["ops"].ekl_tpo_convection(*dev)
+    torch.cuda.synchronize()
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().reshape(3 * E, nv, nv, nv),
+                                            want.reshape(3 * E, nv, nv, nv))
+    assert err.max() <= TOL64, (nq, nv, E, err.max())
 
 
 def test_convection_workload_full_size_sampled(env):

@@ -72,6 +72,24 @@ ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const dou
                                      double* v, int n, long long E, cudaStream_t stream);
 
 /*
+ * The same operator with the pointwise factor formed on the fly instead of read from
+ * memory, for the case where it is a sum of one-dimensional eigenvalues plus a per-element
+ * shift (the paper does not print this variant; it is the structure the inverse
+ * Helmholtz factor has):
+ *
+ *     D[e,i,j,k] = 1 / (((lam[i] + lam[j]) + lam[k]) + c[e])        lam [n], c [E]
+ *
+ * evaluated in exactly this order with IEEE operations, so the result equals
+ * ekl_tpo_inv_helmholtz on the materialised D bit for bit.  Moves 16 n^3 + 8 bytes per
+ * element instead of 24 n^3 and spends n^3 divisions.  fp64, 4 <= n <= 16 (other n:
+ * EKL_TPO_ERR_UNSUPPORTED); even n needs a 16-byte aligned u (EKL_TPO_ERR_ALIGN otherwise).
+ * v == u is allowed.
+ */
+ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, const double* c,
+                                            const double* u, double* v, int n, long long E,
+                                            cudaStream_t stream);
+
+/*
  * Forward rectangular tensor-product operator (the operator family of Eq. 1):
  *
  *     v[e] = (A (x) B (x) C) . u[e],   e = 0..E-1

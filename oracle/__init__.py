@@ -111,6 +111,19 @@ def inv_helmholtz(S, D, u, threads: int = 0) -> np.ndarray:
     return v
 
 
+def lambda_factor(lam, c) -> np.ndarray:
+    """``D[e,i,j,k] = 1/(((lam[i]+lam[j])+lam[k])+c[e])``, the sums taken in this order."""
+    lam, c = _f64(lam), _f64(c)
+    s = (lam[:, None, None] + lam[None, :, None]) + lam[None, None, :]
+    return 1.0 / (s[None, :, :, :] + c[:, None, None, None])
+
+
+def inv_helmholtz_lambda(S, lam, c, u, threads: int = 0) -> np.ndarray:
+    """Inverse Helmholtz whose pointwise factor is given by its eigenvalue sums: the factor is
+    written out with :func:`lambda_factor` and handed to :func:`inv_helmholtz`."""
+    return inv_helmholtz(S, lambda_factor(lam, c), u, threads)
+
+
 def inv_helmholtz_bruteforce(S, D, u) -> np.ndarray:
     """Same operator through the explicit n³×n³ Kronecker matrices (tiny n only)."""
     S, D, u, n, E = _check_ih(S, D, u)

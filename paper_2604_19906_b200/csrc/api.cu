@@ -96,6 +96,28 @@ ekl_tpo_status ekl_tpo_apply_f32(const float* A, const float* B, const float* C,
     return apply_impl<float>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream);
 }
 
+ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, const double* c,
+                                            const double* u, double* v, int n, long long E,
+                                            cudaStream_t stream) {
+    if (n < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
+    if (E == 0) return EKL_TPO_OK;
+    if (!S || !lam || !c || !u || !v) return EKL_TPO_ERR_NULL;
+    if (n < 4 || n > 16) return EKL_TPO_ERR_UNSUPPORTED;
+    if (misaligned(S, 8) || misaligned(lam, 8) || misaligned(c, 8) || misaligned(u, 8) ||
+        misaligned(v, 8) || (n % 2 == 0 && misaligned(u, 16)))
+        return EKL_TPO_ERR_ALIGN;
+    const size_t field = (size_t)E * n * n * n * sizeof(double);
+    if (overlaps(v, field, S, (size_t)n * n * sizeof(double)) ||
+        overlaps(v, field, lam, (size_t)n * sizeof(double)) ||
+        overlaps(v, field, c, (size_t)E * sizeof(double)) ||
+        ((const void*)v != (const void*)u && overlaps(v, field, u, field)))
+        return EKL_TPO_ERR_OVERLAP;
+    cudaError_t err = cudaSuccess;
+    if (!ekl::try_launch_ih_lambda_dmma(S, lam, c, u, v, n, E, stream, &err))
+        return EKL_TPO_ERR_UNSUPPORTED;
+    return err == cudaSuccess ? EKL_TPO_OK : cuda_fail(err);
+}
+
 const char* ekl_tpo_status_string(ekl_tpo_status status) {
     switch (status) {
         case EKL_TPO_OK: return "ok";

@@ -77,6 +77,10 @@ int sm_count();
 template <typename T>
 bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long long E,
                         cudaStream_t stream, cudaError_t* err);
+// Same, with the pointwise factor formed from lam[n] and c[E] instead of read from a field.
+bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double* cvec,
+                               const double* u, double* v, int n, long long E, cudaStream_t stream,
+                               cudaError_t* err);
 template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,

@@ -25,6 +25,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace ekl {
 namespace dmma {
 
@@ -201,16 +203,61 @@ __device__ __forceinline__ void load_factor(double (&d)[SS::kMTiles][2], const T
     }
 }
 
+// Where the pointwise factor of the third inverse-Helmholtz stage comes from.
+struct NoFactor {
+    template <class SS>
+    __device__ __forceinline__ void load(double (&)[SS::kMTiles][2], int, int, int, int) const {}
+};
+
+// a stored field D[e,i,j,k] (natural order), Db pointing at the batch
+template <typename T>
+struct FieldFactor {
+    const T* Db;
+    template <class SS>
+    __device__ __forceinline__ void load(double (&d)[SS::kMTiles][2], int valid_pencils, int warp,
+                                         int slot, int lane) const {
+        load_factor<SS, T>(d, Db, valid_pencils, warp, slot, lane);
+    }
+};
+
+// formed on the fly: 1 / (((lam[i] + lam[j]) + lam[k]) + c[e]), cb pointing at the batch
+struct LambdaFactor {
+    const double* lam;
+    const double* cb;
+    template <class SS>
+    __device__ __forceinline__ void load(double (&d)[SS::kMTiles][2], int valid_pencils, int warp,
+                                         int slot, int lane) const {
+        const int r = lane >> 2, kk = lane & 3;
+        int t;
+        const bool live = tile_live<SS>(warp, slot, t);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int q = 8 * t + 2 * kk + h;
+            const bool ok = live && q < valid_pencils;
+            const int es = ok ? q / SS::kP : 0;
+            const int p = ok ? q - es * SS::kP : 0;
+            const int i = p / SS::E2, j = p - i * SS::E2;
+            const double base = __ldg(lam + i) + __ldg(lam + j);
+            const double ce = __ldg(cb + es);
+#pragma unroll
+            for (int mt = 0; mt < SS::kMTiles; ++mt) {
+                const int o = 8 * mt + r;
+                d[mt][h] = (ok && o < SS::O) ? 1.0 / ((base + __ldg(lam + (o < SS::O ? o : 0))) + ce)
+                                             : 0.0;
+            }
+        }
+    }
+};
+
 // MODE 0: shared -> shared (out).  MODE 1: shared -> shared, times the pointwise factor (dfac
 // holds it for the warp's first tile on entry; later tiles are fetched one tile ahead from
-// Db).  MODE 2: shared -> global (gout, dense, converted to the I/O type T).
+// `fac`).  MODE 2: shared -> global (gout, dense, converted to the I/O type T).
 // `valid_pencils` masks a partly filled batch.  All arithmetic is fp64 whatever T is.
-template <class SS, int MODE, typename T>
+template <class SS, int MODE, typename T, typename Factor>
 __device__ __forceinline__ void run_stage(const double* __restrict__ in, double* __restrict__ out,
                                           T* __restrict__ gout, const OpFrag<SS>& op,
-                                          double (&dfac)[SS::kMTiles][2],
-                                          const T* __restrict__ Db, int valid_pencils, int warp,
-                                          int lane) {
+                                          double (&dfac)[SS::kMTiles][2], const Factor& fac,
+                                          int valid_pencils, int warp, int lane) {
     const int r = lane >> 2, kk = lane & 3;
 #pragma unroll
     for (int slot = 0; slot < SS::kTilesPerWarp; ++slot) {
@@ -234,7 +281,7 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
         }
         double dn[SS::kMTiles][2];
         if (MODE == 1 && slot + 1 < SS::kTilesPerWarp)
-            load_factor<SS, T>(dn, Db, valid_pencils, warp, slot + 1, lane);
+            fac.template load<SS>(dn, valid_pencils, warp, slot + 1, lane);
         double c[SS::kMTiles][2];
 #pragma unroll
         for (int mt = 0; mt < SS::kMTiles; ++mt) {
@@ -383,10 +430,12 @@ struct IhCfg {
 
 // v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])).  T is the type of the fields in memory
 // (double: even N needs 16-byte aligned u; float: widened on load, rounded once on store).
-template <int N, typename T>
+// LAMBDA: the factor is not read from D but formed from lam[N] and c[E] (fp64 only).
+template <int N, typename T, bool LAMBDA = false>
 __global__ void __launch_bounds__(IhCfg<N, T>::kThreads, IhCfg<N, T>::kCtasPerSm)
-inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u, T* v,
-                   long long E) {
+inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
+                   const double* __restrict__ lam, const double* __restrict__ cvec, const T* u,
+                   T* v, long long E) {
     using C = IhCfg<N, T>;
     constexpr bool kBulk = C::kBulk && sizeof(T) == sizeof(double);
     using First = typename C::First;
@@ -437,12 +486,20 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
         const int valid = cnt * kN2;
-        const T* Db = D + e0 * kN3;
+        using Factor = typename std::conditional<LAMBDA, LambdaFactor, FieldFactor<T>>::type;
+        Factor fac;
+        if constexpr (LAMBDA) {
+            fac.lam = lam;
+            fac.cb = cvec + e0;
+        } else {
+            fac.Db = D + e0 * kN3;
+        }
+        const NoFactor none;
         const long long next = batch + gridDim.x;
         if (threadIdx.x == 0 && next < n_batches) {
             const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(T));
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
-            bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
+            if (!LAMBDA) bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
         double dfac[Mid::kMTiles][2];
         if (kBulk) {
@@ -456,18 +513,18 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
             }
         }
         // forward: contract i, j, k
-        run_stage<First, 0, T>(bufA, bufB, nullptr, op, dfac, nullptr, valid, warp, lane);
+        run_stage<First, 0, T>(bufA, bufB, nullptr, op, dfac, none, valid, warp, lane);
         __syncthreads();
         // factor for this warp's first tile of the third stage: a whole stage hides the latency
-        load_factor<Mid, T>(dfac, Db, valid, warp, 0, lane);
-        run_stage<Mid, 0, T>(bufB, bufA, nullptr, op, dfac, nullptr, valid, warp, lane);
+        fac.template load<Mid>(dfac, valid, warp, 0, lane);
+        run_stage<Mid, 0, T>(bufB, bufA, nullptr, op, dfac, none, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 1, T>(bufA, bufB, nullptr, op, dfac, Db, valid, warp, lane);
+        run_stage<Mid, 1, T>(bufA, bufB, nullptr, op, dfac, fac, valid, warp, lane);
         __syncthreads();
         // backward: contract i, j, k with S itself
-        run_stage<Mid, 0, T>(bufB, bufA, nullptr, opb, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0, T>(bufB, bufA, nullptr, opb, dfac, none, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 0, T>(bufA, bufB, nullptr, opb, dfac, nullptr, valid, warp, lane);
+        run_stage<Mid, 0, T>(bufA, bufB, nullptr, opb, dfac, none, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (next < n_batches) {
@@ -484,7 +541,7 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D, const T* u,
                     batch_count(next), bar);
             }
         }
-        run_stage<Last, 2, T>(bufB, nullptr, v + e0 * kN3, opb, dfac, nullptr, valid, warp, lane);
+        run_stage<Last, 2, T>(bufB, nullptr, v + e0 * kN3, opb, dfac, none, valid, warp, lane);
         __syncthreads();
     }
 }
@@ -577,14 +634,14 @@ apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict
         } else {
             wait_copies();
         }
-        run_stage<S1, 0, T>(bufU, bufB, nullptr, opA, none1, nullptr, cnt * S1::kP, warp, lane);
+        run_stage<S1, 0, T>(bufU, bufB, nullptr, opA, none1, NoFactor(), cnt * S1::kP, warp, lane);
         __syncthreads();
         // the landing buffer is free: bring in the next batch under the remaining two stages
         if (next < n_batches) fetch(next);
-        run_stage<S2, 0, T>(bufB, bufA, nullptr, opB, none2, nullptr, cnt * S2::kP, warp, lane);
+        run_stage<S2, 0, T>(bufB, bufA, nullptr, opB, none2, NoFactor(), cnt * S2::kP, warp, lane);
         __syncthreads();
-        run_stage<S3, 2, T>(bufA, nullptr, v + e0 * S3::kOut, opC, none3, nullptr, cnt * S3::kP, warp,
-                            lane);
+        run_stage<S3, 2, T>(bufA, nullptr, v + e0 * S3::kOut, opC, none3, NoFactor(), cnt * S3::kP,
+                            warp, lane);
         // the next batch's first stage writes bufB, which this batch no longer reads
     }
 }

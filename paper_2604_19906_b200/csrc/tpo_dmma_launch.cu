@@ -30,18 +30,20 @@ cudaError_t ctas_per_sm(Kernel kernel, int threads, size_t smem, int (&cached)[6
     return cudaSuccess;
 }
 
-template <int N, typename T>
-cudaError_t launch_ih(const T* S, const T* D, const T* u, T* v, long long E, cudaStream_t stream) {
+template <int N, typename T, bool LAMBDA>
+cudaError_t launch_ih(const T* S, const T* D, const double* lam, const double* cvec, const T* u, T* v,
+                      long long E, cudaStream_t stream) {
     using C = dmma::IhCfg<N, T>;
     static int cached[64] = {0};
     int per_sm = 1;
-    cudaError_t err =
-        ctas_per_sm(dmma::inv_helmholtz_dmma<N, T>, C::kThreads, C::kSmemBytes, cached, &per_sm);
+    cudaError_t err = ctas_per_sm(dmma::inv_helmholtz_dmma<N, T, LAMBDA>, C::kThreads,
+                                  C::kSmemBytes, cached, &per_sm);
     if (err != cudaSuccess) return err;
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
-    dmma::inv_helmholtz_dmma<N, T><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    dmma::inv_helmholtz_dmma<N, T, LAMBDA>
+        <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, lam, cvec, u, v, E);
     return cudaGetLastError();
 }
 
@@ -70,19 +72,19 @@ bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long lo
     // fields are copied in element units, and the L2 prefetches align themselves
     if (sizeof(T) == 8 && n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     switch (n) {
-        case 4: *err = launch_ih<4, T>(S, D, u, v, E, stream); return true;
-        case 5: *err = launch_ih<5, T>(S, D, u, v, E, stream); return true;
-        case 6: *err = launch_ih<6, T>(S, D, u, v, E, stream); return true;
-        case 7: *err = launch_ih<7, T>(S, D, u, v, E, stream); return true;
-        case 8: *err = launch_ih<8, T>(S, D, u, v, E, stream); return true;
-        case 9: *err = launch_ih<9, T>(S, D, u, v, E, stream); return true;
-        case 10: *err = launch_ih<10, T>(S, D, u, v, E, stream); return true;
-        case 11: *err = launch_ih<11, T>(S, D, u, v, E, stream); return true;
-        case 12: *err = launch_ih<12, T>(S, D, u, v, E, stream); return true;
-        case 13: *err = launch_ih<13, T>(S, D, u, v, E, stream); return true;
-        case 14: *err = launch_ih<14, T>(S, D, u, v, E, stream); return true;
-        case 15: *err = launch_ih<15, T>(S, D, u, v, E, stream); return true;
-        case 16: *err = launch_ih<16, T>(S, D, u, v, E, stream); return true;
+        case 4: *err = launch_ih<4, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 5: *err = launch_ih<5, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 6: *err = launch_ih<6, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 7: *err = launch_ih<7, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 8: *err = launch_ih<8, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 9: *err = launch_ih<9, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 10: *err = launch_ih<10, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 11: *err = launch_ih<11, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 12: *err = launch_ih<12, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 13: *err = launch_ih<13, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 14: *err = launch_ih<14, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 15: *err = launch_ih<15, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 16: *err = launch_ih<16, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
         default: return false;
     }
 }
@@ -106,6 +108,33 @@ bool apply_cubic_from(int m, const T* A, const T* B, const T* C, const T* u, T* 
 }
 
 }  // namespace
+
+bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double* cvec,
+                               const double* u, double* v, int n, long long E, cudaStream_t stream,
+                               cudaError_t* err) {
+    if (n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
+    switch (n) {
+#define EKL_LAMBDA_CASE(N_)                                                                 \
+    case N_:                                                                                \
+        *err = launch_ih<N_, double, true>(S, nullptr, lam, cvec, u, v, E, stream);         \
+        return true;
+        EKL_LAMBDA_CASE(4)
+        EKL_LAMBDA_CASE(5)
+        EKL_LAMBDA_CASE(6)
+        EKL_LAMBDA_CASE(7)
+        EKL_LAMBDA_CASE(8)
+        EKL_LAMBDA_CASE(9)
+        EKL_LAMBDA_CASE(10)
+        EKL_LAMBDA_CASE(11)
+        EKL_LAMBDA_CASE(12)
+        EKL_LAMBDA_CASE(13)
+        EKL_LAMBDA_CASE(14)
+        EKL_LAMBDA_CASE(15)
+        EKL_LAMBDA_CASE(16)
+#undef EKL_LAMBDA_CASE
+        default: return false;
+    }
+}
 
 template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,

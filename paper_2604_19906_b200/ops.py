@@ -137,6 +137,29 @@ def ekl_tpo_apply_f32(A, B, C, u, out=None):
     return _apply("ekl_tpo_apply_f32", torch.float32, A, B, C, u, out)
 
 
+def ekl_tpo_inv_helmholtz_lambda(S, lam, c, u, out=None):
+    """Inverse Helmholtz with ``D[e,i,j,k] = 1/(((lam[i]+lam[j])+lam[k])+c[e])`` formed on the
+    fly (fp64, 4 <= n <= 16); bit-identical to :func:`ekl_tpo_inv_helmholtz` on that D."""
+    lib = library()
+    fn = lib.ekl_tpo_inv_helmholtz_lambda
+    fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p]
+    fn.restype = ctypes.c_int
+    E, n = u.shape[0], S.shape[0]
+    if tuple(S.shape) != (n, n) or tuple(u.shape[1:]) != (n, n, n) or tuple(lam.shape) != (n,) \
+            or tuple(c.shape) != (E,):
+        raise ValueError("expected S [n,n], lam [n], c [E], u [E,n,n,n]")
+    dev = u.device
+    if out is None:
+        out = torch.empty_like(u)
+    ptrs = [_dev_ptr(t, nm, torch.float64, dev)
+            for t, nm in ((S, "S"), (lam, "lam"), (c, "c"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = fn(*ptrs, n, E, _stream(dev))
+    if st:
+        raise EklTpoError(st, "ekl_tpo_inv_helmholtz_lambda")
+    return out
+
+
 def ekl_tpo_convection(Dvq, Ivq, M, P, out=None):
     """Volume integral of the convective flux: ``F[c,e] = (I⊗I⊗D)(M∘P[c,0]) + (I⊗D⊗I)(M∘P[c,1])
     + (D⊗I⊗I)(M∘P[c,2])`` in fp64 on the current stream; P is [3,3,E,nq,nq,nq], F [3,E,nv,nv,nv]."""

@@ -296,3 +296,20 @@ def test_convection_special_cases_and_planted_mistakes():
     assert relmax(flat(oracle.convection(Ivq, Dvq, M, P)), ref) > 1e-3          # D and I swapped
     assert relmax(flat(oracle.convection(Dvq, Ivq, M, P[:, ::-1].copy())), ref) > 1e-3  # directions
     assert relmax(flat(oracle.convection(Dvq, Ivq, ones, P)), ref) > 1e-3       # dropped M
+
+
+def test_lambda_factor_matches_its_definition_entry_by_entry():
+    g = rng(77)
+    n, E = 5, 4
+    lam = g.uniform(0.1, 2.0, n)
+    c = g.uniform(0.5, 1.5, E)
+    D = oracle.lambda_factor(lam, c)
+    for e in range(E):
+        for i in range(n):
+            for j in range(n):
+                for k in range(n):
+                    assert D[e, i, j, k] == 1.0 / (((lam[i] + lam[j]) + lam[k]) + c[e])
+    S = g.standard_normal((n, n))
+    u = g.uniform(-1, 1, (E, n, n, n))
+    assert np.array_equal(oracle.inv_helmholtz_lambda(S, lam, c, u), oracle.inv_helmholtz(S, D, u))
+    assert relmax(oracle.inv_helmholtz_lambda(S, lam, c, u), ref_inv_helmholtz_kron(S, D, u)) < 1e-13

@@ -64,7 +64,7 @@ typedef enum {
  *
  * fp64.  `v == u` exactly (in place) is allowed; any other overlap of v with an
  * input is rejected.  1 <= n; n is limited by shared memory (n <= 24 for fp64).
- * Every n from 4 to 16 runs on the FP64 tensor path (for even n this needs a 16-byte
+ * Every n from 4 to 20 runs on the FP64 tensor path (for even n this needs a 16-byte
  * aligned u); every other accepted case runs on a slower general kernel with the same
  * results to rounding.
  */

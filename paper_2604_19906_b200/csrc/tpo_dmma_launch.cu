@@ -85,6 +85,10 @@ bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long lo
         case 14: *err = launch_ih<14, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
         case 15: *err = launch_ih<15, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
         case 16: *err = launch_ih<16, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 17: *err = launch_ih<17, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 18: *err = launch_ih<18, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 19: *err = launch_ih<19, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
+        case 20: *err = launch_ih<20, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
         default: return false;
     }
 }

@@ -250,13 +250,15 @@ struct LambdaFactor {
 };
 
 // MODE 0: shared -> shared (out).  MODE 1: shared -> shared, times the pointwise factor (dfac
-// holds it for the warp's first tile on entry; later tiles are fetched one tile ahead from
-// `fac`).  MODE 2: shared -> global (gout, dense, converted to the I/O type T).
+// holds it for the warp's first FD tiles on entry; the factor of tile i + FD is fetched from
+// `fac` into the registers tile i frees, so a load has FD tiles to arrive: a load that misses
+// L1 takes one to two thousand cycles here, several tiles' worth).  MODE 2: shared -> global
+// (gout, dense, converted to the I/O type T).
 // `valid_pencils` masks a partly filled batch.  All arithmetic is fp64 whatever T is.
-template <class SS, int MODE, typename T, typename Factor>
+template <class SS, int MODE, typename T, typename Factor, int FD = 1>
 __device__ __forceinline__ void run_stage(const double* __restrict__ in, double* __restrict__ out,
                                           T* __restrict__ gout, const OpFrag<SS>& op,
-                                          double (&dfac)[SS::kMTiles][2], const Factor& fac,
+                                          double (&dfac)[FD][SS::kMTiles][2], const Factor& fac,
                                           int valid_pencils, int warp, int lane) {
     const int r = lane >> 2, kk = lane & 3;
 #pragma unroll
@@ -279,9 +281,6 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
             const int repeated = (s > 0) ? SS::k0(s - 1) + 4 - SS::k0(s) : 0;
             b[s] = (kk >= repeated) ? src[SS::k0(s) * SS::IN_PS] : 0.0;
         }
-        double dn[SS::kMTiles][2];
-        if (MODE == 1 && slot + 1 < SS::kTilesPerWarp)
-            fac.template load<SS>(dn, valid_pencils, warp, slot + 1, lane);
         double c[SS::kMTiles][2];
 #pragma unroll
         for (int mt = 0; mt < SS::kMTiles; ++mt) {
@@ -309,17 +308,12 @@ __device__ __forceinline__ void run_stage(const double* __restrict__ in, double*
                     if (MODE == 2)
                         gout[off + o] = (T)c[mt][h];
                     else
-                        out[off + o] = (MODE == 1) ? c[mt][h] * dfac[mt][h] : c[mt][h];
+                        out[off + o] = (MODE == 1) ? c[mt][h] * dfac[slot % FD][mt][h] : c[mt][h];
                 }
             }
         }
-        if (MODE == 1 && slot + 1 < SS::kTilesPerWarp) {
-#pragma unroll
-            for (int mt = 0; mt < SS::kMTiles; ++mt) {
-                dfac[mt][0] = dn[mt][0];
-                dfac[mt][1] = dn[mt][1];
-            }
-        }
+        if (MODE == 1 && slot + FD < SS::kTilesPerWarp)
+            fac.template load<SS>(dfac[slot % FD], valid_pencils, warp, slot + FD, lane);
     }
 }
 
@@ -425,6 +419,9 @@ struct IhCfg {
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
     // bulk copies need 16-byte granules: even N; odd N uses 8-byte asynchronous copies
     static constexpr bool kBulk = (N % 2 == 0);
+    // tiles of the pointwise factor held in registers ahead of their use (measured: deeper
+    // than one pays only where a warp has six or seven tiles per stage)
+    static constexpr int kFactorDepth = (N == 14) ? 3 : (N == 10) ? 2 : 1;
     static_assert(N >= 4, "N >= 4");
 };
 
@@ -501,7 +498,8 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
             if (!LAMBDA) bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
-        double dfac[Mid::kMTiles][2];
+        constexpr int FD = C::kFactorDepth;
+        double dfac[FD][Mid::kMTiles][2];
         if (kBulk) {
             if (!wait_bulk(bar, parity)) break;
             parity ^= 1u;
@@ -513,18 +511,19 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
             }
         }
         // forward: contract i, j, k
-        run_stage<First, 0, T>(bufA, bufB, nullptr, op, dfac, none, valid, warp, lane);
+        run_stage<First, 0, T, NoFactor, FD>(bufA, bufB, nullptr, op, dfac, none, valid, warp, lane);
         __syncthreads();
-        // factor for this warp's first tile of the third stage: a whole stage hides the latency
-        fac.template load<Mid>(dfac, valid, warp, 0, lane);
-        run_stage<Mid, 0, T>(bufB, bufA, nullptr, op, dfac, none, valid, warp, lane);
+        // factor for this warp's first tiles of the third stage: a whole stage hides the latency
+#pragma unroll
+        for (int d = 0; d < FD; ++d) fac.template load<Mid>(dfac[d], valid, warp, d, lane);
+        run_stage<Mid, 0, T, NoFactor, FD>(bufB, bufA, nullptr, op, dfac, none, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 1, T>(bufA, bufB, nullptr, op, dfac, fac, valid, warp, lane);
+        run_stage<Mid, 1, T, Factor, FD>(bufA, bufB, nullptr, op, dfac, fac, valid, warp, lane);
         __syncthreads();
         // backward: contract i, j, k with S itself
-        run_stage<Mid, 0, T>(bufB, bufA, nullptr, opb, dfac, none, valid, warp, lane);
+        run_stage<Mid, 0, T, NoFactor, FD>(bufB, bufA, nullptr, opb, dfac, none, valid, warp, lane);
         __syncthreads();
-        run_stage<Mid, 0, T>(bufA, bufB, nullptr, opb, dfac, none, valid, warp, lane);
+        run_stage<Mid, 0, T, NoFactor, FD>(bufA, bufB, nullptr, opb, dfac, none, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
         if (next < n_batches) {
@@ -541,7 +540,7 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
                     batch_count(next), bar);
             }
         }
-        run_stage<Last, 2, T>(bufB, nullptr, v + e0 * kN3, opb, dfac, none, valid, warp, lane);
+        run_stage<Last, 2, T, NoFactor, FD>(bufB, nullptr, v + e0 * kN3, opb, dfac, none, valid, warp, lane);
         __syncthreads();
     }
 }
@@ -623,7 +622,7 @@ apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict
     };
     if (batch < n_batches) fetch(batch);
     unsigned parity = 0;
-    double none1[S1::kMTiles][2], none2[S2::kMTiles][2], none3[S3::kMTiles][2];
+    double none1[1][S1::kMTiles][2], none2[1][S2::kMTiles][2], none3[1][S3::kMTiles][2];
     for (; batch < n_batches; batch += gridDim.x) {
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);

@@ -3,6 +3,7 @@
 
 #include "dispatch.h"
 #include "tpo_dmma.cuh"
+#include "tpo_tf32.cuh"
 
 namespace ekl {
 namespace {
@@ -47,6 +48,41 @@ cudaError_t launch_ih(const T* S, const T* D, const double* lam, const double* c
     return cudaGetLastError();
 }
 
+// Single precision, split-TF32 tensor path (even extents 8..16, 16-byte aligned u).
+template <int N>
+cudaError_t launch_ih_tf32(const float* S, const float* D, const float* u, float* v, long long E,
+                           cudaStream_t stream) {
+    using C = tf32::IhCfg32<N>;
+    static int cached[64] = {0};
+    int per_sm = 1;
+    cudaError_t err = ctas_per_sm(tf32::inv_helmholtz_tf32<N>, C::kThreads, C::kSmemBytes, cached,
+                                  &per_sm);
+    if (err != cudaSuccess) return err;
+    const long long batches = (E + C::kBe - 1) / C::kBe;
+    long long grid = (long long)sm_count() * per_sm;
+    if (grid > batches) grid = batches;
+    tf32::inv_helmholtz_tf32<N><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    return cudaGetLastError();
+}
+
+bool try_launch_ih_tf32(const float* S, const float* D, const float* u, float* v, int n, long long E,
+                        cudaStream_t stream, cudaError_t* err) {
+    if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+    switch (n) {
+        case 8: *err = launch_ih_tf32<8>(S, D, u, v, E, stream); return true;
+        case 10: *err = launch_ih_tf32<10>(S, D, u, v, E, stream); return true;
+        case 12: *err = launch_ih_tf32<12>(S, D, u, v, E, stream); return true;
+        case 14: *err = launch_ih_tf32<14>(S, D, u, v, E, stream); return true;
+        case 16: *err = launch_ih_tf32<16>(S, D, u, v, E, stream); return true;
+        default: return false;
+    }
+}
+// the fp64 fields have no such path
+bool try_launch_ih_tf32(const double*, const double*, const double*, double*, int, long long,
+                        cudaStream_t, cudaError_t*) {
+    return false;
+}
+
 template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
 cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, long long E,
                       cudaStream_t stream) {
@@ -71,6 +107,7 @@ bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long lo
     // bulk copies of u (fp64, even n) need 16-byte aligned element addresses; odd n and fp32
     // fields are copied in element units, and the L2 prefetches align themselves
     if (sizeof(T) == 8 && n % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
+    if (try_launch_ih_tf32(S, D, u, v, n, E, stream, err)) return true;
     switch (n) {
         case 4: *err = launch_ih<4, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;
         case 5: *err = launch_ih<5, T, false>(S, D, nullptr, nullptr, u, v, E, stream); return true;

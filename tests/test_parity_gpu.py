@@ -88,6 +88,49 @@ def test_inv_helmholtz_f32(env, n, E):
     assert err.max() <= TOL32
 
 
+@pytest.mark.parametrize("n", [8, 10, 12, 14, 16])
+@pytest.mark.parametrize("E", [1, 2, 777, 20001])
+def test_inv_helmholtz_f32_split_tf32_path(env, n, E):
+    """Even extents 8..16 in single precision run on the TF32 tensor path with split operands
+    (three tensor steps per product).  A dropped or wrong cross term would leave an error of
+    1e-4 or more, so the 1e-5 bar is the check; E spans one element, one batch, an odd count
+    and many batches per CTA.  A non-orthogonal, non-symmetric S separates S from its
+    transpose in both halves."""
+    g = rng(900 + n)
+    S = (g.standard_normal((n, n)) / np.sqrt(n)).astype(np.float32)
+    D = g.uniform(0.13, 1.25, (E, n, n, n)).astype(np.float32)
+    u = g.uniform(-1, 1, (E, n, n, n)).astype(np.float32)
+    dS, dD, du = to_dev(env, S), to_dev(env, D), to_dev(env, u)
+    got = env["ops"].ekl_tpo_inv_helmholtz_f32(dS, dD, du)
+    sample = np.unique(np.concatenate([np.arange(min(E, 300)), np.arange(max(E - 300, 0), E)]))
+    want = env["oracle"].inv_helmholtz(S, D[sample], u[sample])
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy()[sample].astype(np.float64), want)
+    assert err.max() <= TOL32, (n, E, err.max())
+    # in place, and the same bits on a second call
+    again = env["ops"].ekl_tpo_inv_helmholtz_f32(dS, dD, du, out=du)
+    assert again.data_ptr() == du.data_ptr()
+    assert env["torch"].equal(again, got)
+
+
+def test_inv_helmholtz_f32_unaligned_u_leaves_the_tf32_path(env):
+    """The TF32 path bulk-copies u and needs it 16-byte aligned; a view that starts 4 bytes
+    into an allocation takes another kernel and must give the same answer to tolerance."""
+    torch = env["torch"]
+    n, E = 14, 37
+    g = rng(4242)
+    S = (g.standard_normal((n, n)) / np.sqrt(n)).astype(np.float32)
+    D = g.uniform(0.13, 1.25, (E, n, n, n)).astype(np.float32)
+    u = g.uniform(-1, 1, (E, n, n, n)).astype(np.float32)
+    flat = torch.empty(E * n ** 3 + 1, dtype=torch.float32, device=env["dev"])
+    du = flat[1:].view(E, n, n, n)
+    du.copy_(torch.from_numpy(u))
+    assert du.data_ptr() % 16 == 4
+    got = env["ops"].ekl_tpo_inv_helmholtz_f32(to_dev(env, S), to_dev(env, D), du)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().astype(np.float64), want)
+    assert err.max() <= TOL32
+
+
 @pytest.mark.parametrize("n", [4, 8, 12, 14])
 def test_inv_helmholtz_exact_special_cases(env, n):
     """S = I gives D∘u bit for bit (every extra term is ×0, +0); a permutation matrix

@@ -260,7 +260,7 @@ def main():
         v = torch.empty_like(case["u"])
         a = (case["S"].data_ptr(), case["D"].data_ptr(), case["u"].data_ptr(), v.data_ptr(),
              wl.n[0], E)
-        fn = lib.ekl_tpo_inv_helmholtz
+        fn = lib.ekl_tpo_inv_helmholtz if wl.dtype == "f64" else lib.ekl_tpo_inv_helmholtz_f32
     elif wl.op == "convection":
         v = torch.empty((3, E) + tuple(wl.m), dtype=torch.float64, device=dev)
         a = (case["Dvq"].data_ptr(), case["Ivq"].data_ptr(), case["M"].data_ptr(),
@@ -321,7 +321,7 @@ def main():
     if base is not None:
         import oracle
         got = (v[:, :ns_oracle].permute(1, 0, 2, 3, 4).contiguous() if wl.op == "convection"
-               else v[:ns_oracle]).cpu().numpy()
+               else v[:ns_oracle]).cpu().numpy().astype(np.float64)
         max_rel_err = float(oracle.rel_err_per_element(got, v_oracle).max())
 
     # ---------------------------------------------------------------- FP64 rate of this device, live
@@ -348,7 +348,7 @@ def main():
 
     # ---------------------------------------------------------------- end to end with host buffers
     e2e = None
-    if not args.no_e2e and wl.op != "convection":
+    if not args.no_e2e and wl.op != "convection" and wl.dtype == "f64":
         e2e = run_e2e(torch, ops, wl, case, dev, stream, args.e2e_steps, world, dist)
 
     if rank != 0:
@@ -365,7 +365,15 @@ def main():
     hbm_peak = float(peaks.get("hbm_gbs", HBM_FALLBACK_GBS))
     t_alu = flops_launch / (FP64_PEAK_TFLOPS * 1e12)
     t_hbm = bytes_launch / (hbm_peak * 1e9)
-    if t_alu >= t_hbm:
+    if wl.dtype == "f32":
+        # single precision runs on the TF32 tensor path, three tensor steps per product; its
+        # peak is the measured bf16 figure times the nominal tf32/bf16 ratio (1.1/2.25)
+        tf32_peak = float(peaks.get("bf16_tflops", 1590.0)) * (1.1 / 2.25)
+        t_alu = 3.0 * flops_launch / (tf32_peak * 1e12)
+    if wl.dtype == "f32" and t_alu >= t_hbm:
+        roof = {"bound": "tensor", "achieved": 3.0 * tf, "peak": tf32_peak, "unit": "TFLOP/s",
+                "frac": 3.0 * tf / tf32_peak}
+    elif t_alu >= t_hbm:
         roof = {"bound": "alu", "achieved": tf, "peak": FP64_PEAK_TFLOPS, "unit": "TFLOP/s",
                 "frac": tf / FP64_PEAK_TFLOPS}
     else:
@@ -378,7 +386,9 @@ def main():
         "algorithmic_bytes": bytes_launch, "algorithmic_flops": flops_launch,
         "kernel_ms": avg_launch_ms,
         "peak_source": ("alu: 148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz; hbm: "
-                        f"MEASURED_PEAKS.json ({peak_src})"),
+                        f"MEASURED_PEAKS.json ({peak_src})" if wl.dtype == "f64" else
+                        f"hbm: MEASURED_PEAKS.json ({peak_src}); tensor: bf16 x 1.1/2.25, "
+                        "three TF32 steps per product"),
         "fp64_tflops": tf, "fp64_peak_derived": FP64_PEAK_TFLOPS,
         "fp64_peak_probe_tflops": fp64_meas,
         "hbm_gbs": gbs, "hbm_peak_gbs": hbm_peak, "hbm_frac": gbs / hbm_peak,

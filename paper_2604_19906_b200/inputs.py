@@ -106,6 +106,9 @@ CONFIGS = (
     # not one of the five stated configurations: the convective-flux integral of Eq. 1 on the
     # paper's batch size (8192 elements per call), 12 quadrature -> 8 volume points
     Workload(5, "convection", (12, 12, 12), (8, 8, 8), 8192),
+    # the largest inverse-Helmholtz configuration with single-precision fields (tolerance 1e-5):
+    # the same streams, rounded to fp32
+    Workload(6, "inv_helmholtz", (14, 14, 14), (14, 14, 14), 131072, "f32"),
 )
 
 
@@ -204,8 +207,12 @@ def host_P(wl: Workload, e0: int, e1: int) -> np.ndarray:
 
 
 def host_case(wl: Workload, e0: int = 0, e1: int | None = None) -> dict:
-    """All inputs of ``wl`` for elements [e0,e1) as NumPy arrays (fp64)."""
+    """All inputs of ``wl`` for elements [e0,e1) as NumPy arrays (fp64; rounded to fp32 for a
+    single-precision workload)."""
     e1 = wl.E if e1 is None else e1
+    if wl.dtype == "f32":
+        wide = host_case(Workload(wl.index, wl.op, wl.n, wl.m, wl.E, "f64"), e0, e1)
+        return {k: (v if k == "lam" else v.astype(np.float32)) for k, v in wide.items()}
     if wl.op == "convection":
         return {"Dvq": gaussian_factor(wl.m[0], wl.n[0], wl.seed, 0),
                 "Ivq": gaussian_factor(wl.m[0], wl.n[0], wl.seed, 1),
@@ -249,6 +256,14 @@ def device_case(wl: Workload, device="cuda:0", e0: int = 0, e1: int | None = Non
     import torch
 
     e1 = wl.E if e1 is None else e1
+    if wl.dtype == "f32":
+        # generated in fp64 by the same kernels, then rounded field by field
+        wide = Workload(wl.index, wl.op, wl.n, wl.m, wl.E, "f64")
+        out = {}
+        for k, t in device_case(wide, device, e0, e1).items():
+            out[k] = t if k == "lam" else t.float()
+            del t
+        return out
     E = e1 - e0
     dev = torch.device(device)
     lib = _fill_lib()

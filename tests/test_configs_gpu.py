@@ -80,3 +80,36 @@ def test_large_configs_sampled(env, idx):
         dmin = case["D"].view(E, -1).abs().amin(dim=1)
         assert bool((nv <= dmax * nu * (1 + 1e-12)).all())
         assert bool((nv >= dmin * nu * (1 - 1e-12)).all())
+
+
+def test_largest_config_in_single_precision_sampled(env):
+    """The largest inverse-Helmholtz configuration with fp32 fields (the TF32 tensor path with
+    split operands), at full size in the launch shape the benchmark times, sampled against the
+    oracle on the same rounded inputs: bar 1e-5 per element."""
+    torch = env["torch"]
+    wl = env["inputs"].CONFIGS[6]
+    assert wl.dtype == "f32" and wl.n == (14, 14, 14) and wl.E == 131072
+    case = env["inputs"].device_case(wl, env["dev"])
+    assert case["u"].dtype == torch.float32
+    got = env["ops"].ekl_tpo_inv_helmholtz_f32(case["S"], case["D"], case["u"])
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(got).all())
+    E = wl.E
+    for e0, e1 in [(0, 96), (E // 2 - 40, E // 2 + 88), (E - 77, E)]:
+        host = env["inputs"].host_case(wl, e0, e1)
+        want = env["oracle"].inv_helmholtz(host["S"], host["D"], host["u"])
+        err = env["oracle"].rel_err_per_element(got[e0:e1].cpu().numpy().astype(np.float64), want)
+        assert err.max() <= 1e-5, (e0, err.max())
+    g = np.random.Generator(np.random.PCG64(906))
+    for e in sorted(g.integers(0, E, size=120).tolist()):
+        host = env["inputs"].host_case(wl, e, e + 1)
+        want = env["oracle"].inv_helmholtz(host["S"], host["D"], host["u"])
+        err = env["oracle"].rel_err_per_element(got[e:e + 1].cpu().numpy().astype(np.float64), want)
+        assert err.max() <= 1e-5, (e, err.max())
+    # both transforms are isometries for the orthogonal S: min|D| ‖u‖ <= ‖v‖ <= max|D| ‖u‖
+    nu = torch.linalg.vector_norm(case["u"].double().view(E, -1), dim=1)
+    nv = torch.linalg.vector_norm(got.double().view(E, -1), dim=1)
+    dmax = case["D"].double().view(E, -1).abs().amax(dim=1)
+    dmin = case["D"].double().view(E, -1).abs().amin(dim=1)
+    assert bool((nv <= dmax * nu * (1 + 1e-5)).all())
+    assert bool((nv >= dmin * nu * (1 - 1e-5)).all())

@@ -137,7 +137,11 @@ ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const do
  * the rest) and accumulated in fp32, the fields stay fp32 on chip; measured error about 4e-7.
  * On the FP64 tensor path (the other extents from 4 to 20, and ekl_tpo_apply_f32) the fields
  * are widened to fp64 on chip, all arithmetic is fp64, and v is rounded to fp32 once when it
- * is stored; the general kernel computes in fp32.
+ * is stored; the general kernel computes in fp32.  With EKL_TPO_F32_PATH=tcgen05 in the
+ * environment (read once, at the first call) the split-TF32 case runs on tcgen05.mma with the
+ * accumulator in tensor memory instead: same results to tolerance, slower on this operator
+ * (kept for comparison); it needs D and v 8-byte aligned and holds 32 columns of tensor memory
+ * per CTA while it runs.
  */
 ekl_tpo_status ekl_tpo_inv_helmholtz_f32(const float* S, const float* D, const float* u,
                                          float* v, int n, long long E, cudaStream_t stream);

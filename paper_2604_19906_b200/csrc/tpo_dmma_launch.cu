@@ -4,6 +4,10 @@
 #include "dispatch.h"
 #include "tpo_dmma.cuh"
 #include "tpo_tf32.cuh"
+#include "tpo_umma.cuh"
+
+#include <cstdlib>
+#include <cstring>
 
 namespace ekl {
 namespace {
@@ -65,9 +69,55 @@ cudaError_t launch_ih_tf32(const float* S, const float* D, const float* u, float
     return cudaGetLastError();
 }
 
+// The same operator on the asynchronous tensor path (tcgen05.mma, accumulator in tensor memory).
+// It is correct but slower here (the 16-column operator makes every tensor instruction re-read
+// its 128-row operand from shared memory), so it only runs when EKL_TPO_F32_PATH=tcgen05 asks
+// for it (A/B measurements).
+template <int N>
+cudaError_t launch_ih_umma(const float* S, const float* D, const float* u, float* v, long long E,
+                           cudaStream_t stream) {
+    using C = umma::Cfg<N>;
+    static bool ready[64] = {false};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!ready[dev]) {
+        err = cudaFuncSetAttribute(umma::inv_helmholtz_umma<N>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+        if (err != cudaSuccess) return err;
+        ready[dev] = true;
+    }
+    // as many CTAs as shared memory lets an SM hold (the occupancy query answers 1 for kernels
+    // that allocate tensor memory; more do run side by side, 32 columns each)
+    long long grid = (long long)sm_count() * C::kCtasPerSm;
+    if (grid > E) grid = E;
+    umma::inv_helmholtz_umma<N><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    return cudaGetLastError();
+}
+
+static bool f32_path_is_tcgen05() {
+    static const bool on = [] {
+        const char* p = std::getenv("EKL_TPO_F32_PATH");
+        return p && std::strcmp(p, "tcgen05") == 0;
+    }();
+    return on;
+}
+
 bool try_launch_ih_tf32(const float* S, const float* D, const float* u, float* v, int n, long long E,
                         cudaStream_t stream, cudaError_t* err) {
     if (reinterpret_cast<uintptr_t>(u) % 16) return false;
+    if (f32_path_is_tcgen05() && reinterpret_cast<uintptr_t>(D) % 8 == 0 &&
+        reinterpret_cast<uintptr_t>(v) % 8 == 0) {
+        switch (n) {
+            case 8: *err = launch_ih_umma<8>(S, D, u, v, E, stream); return true;
+            case 10: *err = launch_ih_umma<10>(S, D, u, v, E, stream); return true;
+            case 12: *err = launch_ih_umma<12>(S, D, u, v, E, stream); return true;
+            case 14: *err = launch_ih_umma<14>(S, D, u, v, E, stream); return true;
+            case 16: *err = launch_ih_umma<16>(S, D, u, v, E, stream); return true;
+            default: break;
+        }
+    }
     switch (n) {
         case 8: *err = launch_ih_tf32<8>(S, D, u, v, E, stream); return true;
         case 10: *err = launch_ih_tf32<10>(S, D, u, v, E, stream); return true;

@@ -132,10 +132,11 @@ ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const do
 /*
  * Single-precision twins of ekl_tpo_inv_helmholtz and ekl_tpo_apply (same layout and
  * rules; tolerance 1e-5 instead of 1e-12).  ekl_tpo_inv_helmholtz_f32 with an even n from 8
- * to 16 and a 16-byte aligned u runs on the TF32 tensor path with split operands: every
+ * to 16, and ekl_tpo_apply_f32 for cubic n -> m with even n, m from 8 to 16, both with a
+ * 16-byte aligned u, run on the TF32 tensor path with split operands: every
  * product is taken as a_hi*b_hi + a_lo*b_hi + a_hi*b_lo (hi = the value rounded to TF32, lo =
  * the rest) and accumulated in fp32, the fields stay fp32 on chip; measured error about 4e-7.
- * On the FP64 tensor path (the other extents from 4 to 20, and ekl_tpo_apply_f32) the fields
+ * On the FP64 tensor path (the other extents from 4 to 20, the other cubic pairs) the fields
  * are widened to fp64 on chip, all arithmetic is fp64, and v is rounded to fp32 once when it
  * is stored; the general kernel computes in fp32.  With EKL_TPO_F32_PATH=tcgen05 in the
  * environment (read once, at the first call) the split-TF32 case runs on tcgen05.mma with the

@@ -133,6 +133,52 @@ bool try_launch_ih_tf32(const double*, const double*, const double*, double*, in
     return false;
 }
 
+// Forward operator, single precision, split-TF32 tensor path (cubic n -> m, even extents 8..16).
+template <int N, int M>
+cudaError_t launch_ap_tf32(const float* A, const float* B, const float* Cm, const float* u, float* v,
+                           long long E, cudaStream_t stream) {
+    using C = tf32::ApplyCfg32<N, N, N, M, M, M>;
+    auto kernel = tf32::apply_tf32<N, N, N, M, M, M>;
+    static int cached[64] = {0};
+    int per_sm = 1;
+    cudaError_t err = ctas_per_sm(kernel, C::kThreads, C::kSmemBytes, cached, &per_sm);
+    if (err != cudaSuccess) return err;
+    const long long batches = (E + C::kBe - 1) / C::kBe;
+    long long grid = (long long)sm_count() * per_sm;
+    if (grid > batches) grid = batches;
+    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E);
+    return cudaGetLastError();
+}
+
+template <int N>
+bool apply_tf32_from(int m, const float* A, const float* B, const float* C, const float* u, float* v,
+                     long long E, cudaStream_t stream, cudaError_t* err) {
+    switch (m) {
+        case 8: *err = launch_ap_tf32<N, 8>(A, B, C, u, v, E, stream); return true;
+        case 10: *err = launch_ap_tf32<N, 10>(A, B, C, u, v, E, stream); return true;
+        case 12: *err = launch_ap_tf32<N, 12>(A, B, C, u, v, E, stream); return true;
+        case 14: *err = launch_ap_tf32<N, 14>(A, B, C, u, v, E, stream); return true;
+        case 16: *err = launch_ap_tf32<N, 16>(A, B, C, u, v, E, stream); return true;
+        default: return false;
+    }
+}
+
+bool try_launch_apply_tf32(const float* A, const float* B, const float* C, const float* u, float* v,
+                           int n, int m, long long E, cudaStream_t stream, cudaError_t* err) {
+    switch (n) {
+        case 8: return apply_tf32_from<8>(m, A, B, C, u, v, E, stream, err);
+        case 10: return apply_tf32_from<10>(m, A, B, C, u, v, E, stream, err);
+        case 12: return apply_tf32_from<12>(m, A, B, C, u, v, E, stream, err);
+        case 14: return apply_tf32_from<14>(m, A, B, C, u, v, E, stream, err);
+        case 16: return apply_tf32_from<16>(m, A, B, C, u, v, E, stream, err);
+        default: return false;
+    }
+}
+bool try_launch_apply_tf32(const double*, const double*, const double*, const double*, double*, int,
+                           int, long long, cudaStream_t, cudaError_t*) {
+    return false;
+}
+
 template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
 cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, long long E,
                       cudaStream_t stream) {
@@ -234,6 +280,7 @@ bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v,
     // fp64 u is bulk-copied plane by plane: 16-byte aligned element addresses
     if (sizeof(T) == 8 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) return false;
+    if (try_launch_apply_tf32(A, B, C, u, v, n0, m0, E, stream, err)) return true;
     switch (n0) {
         case 4: return apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err);
         case 6: return apply_cubic_from<6, T>(m0, A, B, C, u, v, E, stream, err);

@@ -288,5 +288,102 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
     }
 }
 
+// ------------------------------------------------------------------ forward rectangular operator
+
+template <int N0, int N1, int N2, int M0, int M1, int M2>
+struct ApplyCfg32 {
+    static_assert(N0 >= 8 && N1 >= 8 && N2 >= 8 && M0 <= 16 && M1 <= 16 && M2 <= 16,
+                  "contraction extents from 8, output extents up to 16");
+    // u as it lands: [n0][n1*n2] with padded planes
+    static constexpr int kPS0 = pad_plane32(N1 * N2), kES0 = N0 * kPS0;
+    // after the first stage: [n1][n2][m0]
+    static constexpr int kRS1 = pad_row32(M0), kPS1 = pad_plane32(N2 * kRS1), kES1 = N1 * kPS1;
+    // after the second stage: [n2][m0][m1]
+    static constexpr int kRS2 = pad_row32(M1), kPS2 = pad_plane32(M0 * kRS2), kES2 = N2 * kPS2;
+    static constexpr int kBe = 2;
+    static constexpr int kMaxTiles =
+        kBe * (N1 * N2 > N2 * M0 ? (N1 * N2 > M0 * M1 ? N1 * N2 : M0 * M1)
+                                 : (N2 * M0 > M0 * M1 ? N2 * M0 : M0 * M1)) / 8;
+    static constexpr int kWarps = (kMaxTiles > 32) ? 8 : 4;
+    using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
+    using S2 = Stage<N1, M1, N2, M0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
+    using S3 = Stage<N2, M2, M0, M1, kBe, kWarps, kRS2, kPS2, kES2, M2, M1 * M2, M0 * M1 * M2>;
+    static constexpr int kThreads = 32 * kWarps;
+    static constexpr int kU = kBe * kES0, kB = kBe * kES1, kA = kBe * kES2;
+    static constexpr size_t kSmemBytes = (size_t)(kU + kB + kA) * sizeof(float) + 16;
+    static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
+#ifndef EKL_TF32_APPLY_MAX_WARPS
+#define EKL_TF32_APPLY_MAX_WARPS EKL_TF32_MAX_WARPS
+#endif
+    static constexpr int kByWarps = EKL_TF32_APPLY_MAX_WARPS / kWarps;
+    static constexpr int kCtasPerSm =
+        (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
+    static_assert((N1 * N2) % 4 == 0, "planes must be a whole number of 16-byte units");
+};
+
+// v[e] = (A(x)B(x)C) u[e], fp32 fields; contraction order A, B, C (slowest axis first); u must
+// be 16-byte aligned.
+template <int N0, int N1, int N2, int M0, int M1, int M2>
+__global__ void __launch_bounds__(ApplyCfg32<N0, N1, N2, M0, M1, M2>::kThreads,
+                                  ApplyCfg32<N0, N1, N2, M0, M1, M2>::kCtasPerSm)
+apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float* __restrict__ Cm,
+           const float* __restrict__ u, float* __restrict__ v, long long E) {
+    using C = ApplyCfg32<N0, N1, N2, M0, M1, M2>;
+    using S1 = typename C::S1;
+    using S2 = typename C::S2;
+    using S3 = typename C::S3;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* bufU = reinterpret_cast<float*>(smem_raw);
+    float* bufB = bufU + C::kU;
+    float* bufA = bufB + C::kB;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(bufA + C::kA);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = ((threadIdx.x >> 5) + blockIdx.x) % C::kWarps;
+
+    // all three operators, split, stay in registers for the life of the CTA
+    OpFrag32<Steps8<N0>::kSteps> opA;
+    OpFrag32<Steps8<N1>::kSteps> opB;
+    OpFrag32<Steps8<N2>::kSteps> opC;
+    load_op32<S1>(opA, A, true, lane);
+    load_op32<S2>(opB, B, true, lane);
+    load_op32<S3>(opC, Cm, true, lane);
+
+    const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    if (threadIdx.x == 0) dmma::mbar_init(bar, 1);
+    __syncthreads();
+    auto batch_count = [&](long long b) {
+        const long long e0 = b * C::kBe;
+        return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
+    };
+    auto fetch = [&](long long b) {
+        if (threadIdx.x == 0) {
+            dmma::fence_async_proxy();
+            load_elements32<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + b * C::kBe * S1::kIn,
+                                                           batch_count(b), bar);
+        }
+    };
+    long long batch = blockIdx.x;
+    if (batch < n_batches) fetch(batch);
+    unsigned parity = 0;
+    float none[1][4];
+    for (; batch < n_batches; batch += gridDim.x) {
+        const long long e0 = batch * C::kBe;
+        const int cnt = batch_count(batch);
+        const long long next = batch + gridDim.x;
+        if (!dmma::wait_bulk(bar, parity)) break;
+        parity ^= 1u;
+        run_stage32<S1, 0, 1>(bufU, bufB, nullptr, opA, none, nullptr, cnt * S1::kP, warp, lane);
+        __syncthreads();
+        // the landing buffer is free: bring in the next batch under the remaining two stages
+        if (next < n_batches) fetch(next);
+        run_stage32<S2, 0, 1>(bufB, bufA, nullptr, opB, none, nullptr, cnt * S2::kP, warp, lane);
+        __syncthreads();
+        run_stage32<S3, 2, 1>(bufA, nullptr, v + e0 * S3::kOut, opC, none, nullptr, cnt * S3::kP, warp,
+                              lane);
+        // the next batch's first stage writes bufB, which this batch no longer reads
+    }
+}
+
 }  // namespace tf32
 }  // namespace ekl

@@ -292,6 +292,22 @@ def test_apply_f32(env, nn, mm):
     assert err.max() <= TOL32
 
 
+@pytest.mark.parametrize("n", [8, 10, 12, 14, 16])
+@pytest.mark.parametrize("m", [8, 10, 12, 14, 16])
+def test_apply_f32_split_tf32_path(env, n, m):
+    """Cubic n -> m forward operators with even extents 8..16 in single precision run on the
+    TF32 tensor path with split operands; three different matrices separate the axes, an odd
+    element count leaves a partly filled batch."""
+    g = rng(3000 + 20 * n + m)
+    E = 515
+    A, B, C = ((g.standard_normal((m, n)) / np.sqrt(n)).astype(np.float32) for _ in range(3))
+    u = g.uniform(-1, 1, (E, n, n, n)).astype(np.float32)
+    got = env["ops"].ekl_tpo_apply_f32(*(to_dev(env, x) for x in (A, B, C, u)))
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().astype(np.float64), want)
+    assert err.max() <= TOL32, (n, m, err.max())
+
+
 def test_apply_selection_matrices_gather_exactly(env):
     g = rng(8)
     nn, mm = (8, 8, 8), (12, 12, 12)

@@ -47,7 +47,7 @@ HBM_FALLBACK_GBS = 6650.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per element of the operator
 # kernel, from the ncu captures summarised under profiles/ (taken on a smaller E of the same
 # kernel; traffic is proportional to the number of elements).  Workload index -> bytes.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {3: 67676.0, 4: 16200.0, 6: 32590.0}
+NCU_TRAFFIC_BYTES_PER_ELEMENT = {3: 67676.0, 4: 16200.0, 5: 150400.0, 6: 32590.0}
 
 
 def measured_peaks():

@@ -395,7 +395,11 @@ struct IhCfg {
     // elements per batch: two (four for the smallest) unless that leaves room for one CTA only
     static constexpr int kBe = (N <= 6) ? 4 : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
-    static constexpr int kWarps = (N == 14)           ? 8
+    // warps per CTA: an even deal of the tiles where one exists, with the measured exceptions
+    // (CTAs of 5 warps load the four scheduler partitions 2,1,1,1: n = 10 and 20 run 8 % and
+    // 26 % faster with 4 and 8 warps, n = 17 12 % faster with 4)
+    static constexpr int kWarps = (N == 14 || N == 20) ? 8
+                                  : (N == 10 || N == 17) ? 4
                                   : (kTiles <= 36 && kTiles % 4 == 0) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6

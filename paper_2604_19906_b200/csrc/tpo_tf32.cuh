@@ -308,7 +308,10 @@ struct ApplyCfg32 {
     static constexpr int kMaxTiles =
         kBe * (N1 * N2 > N2 * M0 ? (N1 * N2 > M0 * M1 ? N1 * N2 : M0 * M1)
                                  : (N2 * M0 > M0 * M1 ? N2 * M0 : M0 * M1)) / 8;
-    static constexpr int kWarps = (kMaxTiles > 32) ? 8 : 4;
+#ifndef EKL_TF32_APPLY_TILES_FOR_8
+#define EKL_TF32_APPLY_TILES_FOR_8 48
+#endif
+    static constexpr int kWarps = (kMaxTiles > EKL_TF32_APPLY_TILES_FOR_8) ? 8 : 4;
     using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
     using S2 = Stage<N1, M1, N2, M0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
     using S3 = Stage<N2, M2, M0, M1, kBe, kWarps, kRS2, kPS2, kES2, M2, M1 * M2, M0 * M1 * M2>;

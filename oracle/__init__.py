@@ -14,6 +14,8 @@ Operators (row-major arrays, element index slowest, see ``tpo_oracle.c``):
 
 * ``inv_helmholtz(S, D, u)``: ``v_e = (S⊗S⊗S)·(D_e ∘ ((Sᵀ⊗Sᵀ⊗Sᵀ)·u_e))`` with the
   lifted (sum-factorised) reductions of Section 5.2 of the paper.
+* ``inv_helmholtz3(S0, S1, S2, D, u)``: the same with one operator and one extent per
+  direction, ``v_e = (S0⊗S1⊗S2)·(D_e ∘ ((S0ᵀ⊗S1ᵀ⊗S2ᵀ)·u_e))`` (per-direction matrices as in Eq. 1).
 * ``tpo_apply(A, B, C, u)``: ``v_e = (A⊗B⊗C)·u_e``, rectangular factors, the
   operator family of Eq. 1.
 * ``convection(Dvq, Ivq, M, P)``: the volume integral of the convective flux, Eq. 1.
@@ -67,6 +69,10 @@ def _load():
         lib.oracle_tpo_apply_ld.argtypes = [dp, dp, dp, dp, dp, i, i, i, i, i, i, ll]
         lib.oracle_convection_f64.argtypes = [dp, dp, dp, dp, dp, i, i, ll, i]
         lib.oracle_convection_bruteforce_f64.argtypes = [dp, dp, dp, dp, dp, i, i, ll]
+        lib.oracle_inv_helmholtz3_f64.argtypes = [dp, dp, dp, dp, dp, dp, i, i, i, ll, i]
+        lib.oracle_inv_helmholtz3_bruteforce_f64.argtypes = [dp, dp, dp, dp, dp, dp, i, i, i, ll]
+        lib.oracle_inv_helmholtz3_f64.restype = i
+        lib.oracle_inv_helmholtz3_bruteforce_f64.restype = i
         lib.oracle_convection_f64.restype = i
         lib.oracle_convection_bruteforce_f64.restype = i
         for f in (lib.oracle_inv_helmholtz_f64, lib.oracle_inv_helmholtz_bruteforce_f64,
@@ -122,6 +128,40 @@ def inv_helmholtz_lambda(S, lam, c, u, threads: int = 0) -> np.ndarray:
     """Inverse Helmholtz whose pointwise factor is given by its eigenvalue sums: the factor is
     written out with :func:`lambda_factor` and handed to :func:`inv_helmholtz`."""
     return inv_helmholtz(S, lambda_factor(lam, c), u, threads)
+
+
+def _check_ih3(S0, S1, S2, D, u):
+    S0, S1, S2, D, u = _f64(S0), _f64(S1), _f64(S2), _f64(D), _f64(u)
+    for S in (S0, S1, S2):
+        if S.ndim != 2 or S.shape[0] != S.shape[1]:
+            raise ValueError("S0, S1, S2 must be square matrices")
+    nn = (S0.shape[0], S1.shape[0], S2.shape[0])
+    if u.ndim != 4 or u.shape[1:] != nn or D.shape != u.shape:
+        raise ValueError("D and u must be [E,n0,n1,n2] with n_d the order of S_d")
+    return S0, S1, S2, D, u, nn, u.shape[0]
+
+
+def inv_helmholtz3(S0, S1, S2, D, u, threads: int = 0) -> np.ndarray:
+    """Inverse Helmholtz with one operator and one extent per direction:
+    ``v_e = (S0⊗S1⊗S2)·(D_e ∘ ((S0ᵀ⊗S1ᵀ⊗S2ᵀ)·u_e))``, S0 on the slowest in-element axis."""
+    S0, S1, S2, D, u, nn, E = _check_ih3(S0, S1, S2, D, u)
+    v = np.empty_like(u)
+    if E and _load().oracle_inv_helmholtz3_f64(_ptr(S0), _ptr(S1), _ptr(S2), _ptr(D), _ptr(u),
+                                               _ptr(v), *nn, E, int(threads)):
+        raise MemoryError("oracle scratch allocation failed")
+    return v
+
+
+def inv_helmholtz3_bruteforce(S0, S1, S2, D, u) -> np.ndarray:
+    """The same operator through the explicit Kronecker matrices (tiny extents only)."""
+    S0, S1, S2, D, u, nn, E = _check_ih3(S0, S1, S2, D, u)
+    if np.prod(nn) > 256:
+        raise ValueError("brute force is meant for tiny shapes")
+    v = np.empty_like(u)
+    if E and _load().oracle_inv_helmholtz3_bruteforce_f64(_ptr(S0), _ptr(S1), _ptr(S2), _ptr(D),
+                                                          _ptr(u), _ptr(v), *nn, E):
+        raise MemoryError("oracle scratch allocation failed")
+    return v
 
 
 def inv_helmholtz_bruteforce(S, D, u) -> np.ndarray:

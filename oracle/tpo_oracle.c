@@ -162,6 +162,57 @@ int oracle_inv_helmholtz_f64(const double *S, const double *D, const double *u,
 }
 
 /*
+ * Inverse Helmholtz with one operator per direction and its own extent per direction
+ * (the per-direction matrices of Eq. 1 and of the convective-flux listing, where every
+ * axis has its own small matrix), all E elements:
+ *   v[e] = (S0 (x) S1 (x) S2) ( D[e] o ( (S0^T (x) S1^T (x) S2^T) u[e] ) ).
+ * S0:[n0,n0] acts on the slowest in-element axis, S2:[n2,n2] on the contiguous one;
+ * D,u,v:[E,n0,n1,n2].
+ */
+static double *transposed(const double *S, int n)
+{
+    double *St = (double *)malloc((size_t)n * n * sizeof(double) + 8);
+    if (!St) return NULL;
+    for (int a = 0; a < n; ++a)
+        for (int b = 0; b < n; ++b)
+            St[a * n + b] = S[b * n + a];
+    return St;
+}
+
+int oracle_inv_helmholtz3_f64(const double *S0, const double *S1, const double *S2,
+                              const double *D, const double *u, double *v,
+                              int n0, int n1, int n2, long long E, int threads)
+{
+    const size_t n3 = (size_t)n0 * n1 * n2;
+    int fail = 0;
+    double *St0 = transposed(S0, n0), *St1 = transposed(S1, n1), *St2 = transposed(S2, n2);
+    if (!St0 || !St1 || !St2) { free(St0); free(St1); free(St2); return -1; }
+    threads = pick_threads(threads);
+#pragma omp parallel num_threads(threads)
+    {
+        double *p = (double *)malloc((3 * n3 + 1) * sizeof(double));
+        if (!p) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+            double *q = p + n3, *t = q + n3;
+#pragma omp for schedule(static)
+            for (long long e = 0; e < E; ++e) {
+                const double *ue = u + (size_t)e * n3, *De = D + (size_t)e * n3;
+                apply_one(St0, St1, St2, ue, t, p, q, n0, n1, n2, n0, n1, n2);
+                for (size_t x = 0; x < n3; ++x) t[x] = De[x] * t[x];
+                apply_one(S0, S1, S2, t, v + (size_t)e * n3, p, q, n0, n1, n2, n0, n1, n2);
+            }
+        }
+        free(p);
+    }
+    free(St0); free(St1); free(St2);
+    return fail ? -1 : 0;
+}
+
+/*
  * Volume integral of the convective flux (Eq. 1 of the paper and its one-statement
  * listing), sum-factorised term by term:
  *
@@ -307,6 +358,32 @@ int oracle_inv_helmholtz_bruteforce_f64(const double *S, const double *D, const 
     }
     free(K1); free(K2); free(St); free(t);
     return 0;
+}
+
+/* v[e] = K2 diag(vec D[e]) K1 vec(u[e]),  K1 = kron(S0^T,S1^T,S2^T), K2 = kron(S0,S1,S2). */
+int oracle_inv_helmholtz3_bruteforce_f64(const double *S0, const double *S1, const double *S2,
+                                         const double *D, const double *u, double *v,
+                                         int n0, int n1, int n2, long long E)
+{
+    const size_t n3 = (size_t)n0 * n1 * n2;
+    double *St0 = transposed(S0, n0), *St1 = transposed(S1, n1), *St2 = transposed(S2, n2);
+    double *t = (double *)malloc(n3 * sizeof(double) + 8);
+    double *K1 = NULL, *K2 = NULL;
+    int rc = -1;
+    if (St0 && St1 && St2 && t) {
+        K1 = kron3(St0, St1, St2, n0, n1, n2, n0, n1, n2);
+        K2 = kron3(S0, S1, S2, n0, n1, n2, n0, n1, n2);
+    }
+    if (K1 && K2) {
+        for (long long e = 0; e < E; ++e) {
+            matvec(K1, u + (size_t)e * n3, t, n3, n3);
+            for (size_t x = 0; x < n3; ++x) t[x] = D[(size_t)e * n3 + x] * t[x];
+            matvec(K2, t, v + (size_t)e * n3, n3, n3);
+        }
+        rc = 0;
+    }
+    free(K1); free(K2); free(St0); free(St1); free(St2); free(t);
+    return rc;
 }
 
 /* ---- extended-precision re-evaluation (accuracy level of the oracle) ----- */

@@ -30,6 +30,17 @@ def inv_helmholtz_int(S, D, u, n):
     return [[[v[i, j, k] for k in rng] for j in rng] for i in rng]
 
 
+def inv_helmholtz3_int(S0, S1, S2, D, u, nn):
+    """One operator per direction: forward stage S0^T, S1^T, S2^T, backward stage S0, S1, S2."""
+    idx = list(itertools.product(range(nn[0]), range(nn[1]), range(nn[2])))
+    t = {(i, j, k): sum(S0[l][i] * S1[m][j] * S2[q][k] * u[l][m][q] for l, m, q in idx)
+         for i, j, k in idx}
+    r = {x: D[x[0]][x[1]][x[2]] * t[x] for x in idx}
+    v = {(i, j, k): sum(S0[i][l] * S1[j][m] * S2[k][q] * r[l, m, q] for l, m, q in idx)
+         for i, j, k in idx}
+    return [[[v[i, j, k] for k in range(nn[2])] for j in range(nn[1])] for i in range(nn[0])]
+
+
 def apply_int(A, B, C, u, nn, mm):
     return [[[sum(A[i][l] * B[j][m] * C[k][q] * u[l][m][q]
                   for l in range(nn[0]) for m in range(nn[1]) for q in range(nn[2]))
@@ -86,6 +97,23 @@ def main():
           "# v = (A(x)B(x)C) u, Kronecker ordering of Eq. 1: A <-> slowest in-element axis,\n"
           "# C <-> contiguous axis; exact integers\n",
           [("nn", nn), ("mm", mm), ("A", flat(A)), ("B", flat(B)), ("C", flat(C)),
+           ("u", flat(u)), ("v", flat(v))])
+
+    # inverse Helmholtz with one operator and one extent per direction (per-direction
+    # matrices as in Eq. 1): three different non-symmetric matrices, extents 2, 3, 4
+    nn = (2, 3, 4)
+    S0 = [[2, -1], [3, 1]]
+    S1 = [[1, 0, -2], [2, 1, 1], [-1, 3, 0]]
+    S2 = [[((a * 4 + b) * 3 % 7) - 3 for b in range(4)] for a in range(4)]
+    D = [[[((2 * i + 3 * j + 5 * k) % 7) - 3 for k in range(nn[2])] for j in range(nn[1])]
+         for i in range(nn[0])]
+    u = [[[((i * 12 + j * 4 + k) * 5 % 9) - 4 for k in range(nn[2])] for j in range(nn[1])]
+         for i in range(nn[0])]
+    v = inv_helmholtz3_int(S0, S1, S2, D, u, nn)
+    write("inv_helmholtz3_2x3x4_int.txt",
+          "# v = (S0(x)S1(x)S2)(D o ((S0^T(x)S1^T(x)S2^T) u)), S0 <-> slowest in-element axis,\n"
+          "# S2 <-> contiguous axis; exact integers\n",
+          [("nn", nn), ("S0", flat(S0)), ("S1", flat(S1)), ("S2", flat(S2)), ("D", flat(D)),
            ("u", flat(u)), ("v", flat(v))])
 
 

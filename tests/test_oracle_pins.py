@@ -313,3 +313,89 @@ def test_lambda_factor_matches_its_definition_entry_by_entry():
     u = g.uniform(-1, 1, (E, n, n, n))
     assert np.array_equal(oracle.inv_helmholtz_lambda(S, lam, c, u), oracle.inv_helmholtz(S, D, u))
     assert relmax(oracle.inv_helmholtz_lambda(S, lam, c, u), ref_inv_helmholtz_kron(S, D, u)) < 1e-13
+
+
+# ------------------------------------------------------------------ one operator per direction
+
+def ref_inv_helmholtz3_kron(S0, S1, S2, D, u):
+    """numpy.kron (library routine): K2 diag(D) K1 with K1 = S0ᵀ⊗S1ᵀ⊗S2ᵀ, K2 = S0⊗S1⊗S2."""
+    E = u.shape[0]
+    K1 = np.kron(np.kron(S0.T, S1.T), S2.T)
+    K2 = np.kron(np.kron(S0, S1), S2)
+    t = (K1 @ u.reshape(E, -1).T).T * D.reshape(E, -1)
+    return (K2 @ t.T).T.reshape(u.shape)
+
+
+@pytest.mark.parametrize("nn", [(2, 3, 4), (4, 2, 3), (1, 5, 2), (3, 3, 3), (5, 1, 1)])
+def test_inv_helmholtz3_matches_numpy_kron_and_einsum(nn):
+    g = rng(500 + 100 * nn[0] + 10 * nn[1] + nn[2])
+    S0, S1, S2 = (g.standard_normal((n, n)) for n in nn)      # three different, non-symmetric
+    D = g.uniform(0.1, 1.3, (3,) + nn)
+    u = g.uniform(-1, 1, (3,) + nn)
+    ref = ref_inv_helmholtz3_kron(S0, S1, S2, D, u)
+    got = oracle.inv_helmholtz3(S0, S1, S2, D, u)
+    assert relmax(got, ref) < 1e-13
+    assert relmax(oracle.inv_helmholtz3_bruteforce(S0, S1, S2, D, u), ref) < 1e-13
+    ein = np.einsum("il,jm,kn,elmn->eijk", S0, S1, S2,
+                    D * np.einsum("li,mj,nk,elmn->eijk", S0, S1, S2, u))
+    assert relmax(got, ein) < 1e-13
+
+
+def test_inv_helmholtz3_golden_integer_fixture_is_reproduced_exactly():
+    g = read_golden("inv_helmholtz3_2x3x4_int.txt")
+    nn = tuple(int(x) for x in g["nn"])
+    S0, S1, S2 = (g[f"S{d}"].reshape(nn[d], nn[d]) for d in range(3))
+    D = g["D"].reshape((1,) + nn)
+    u = g["u"].reshape((1,) + nn)
+    want = g["v"].reshape((1,) + nn)
+    assert np.array_equal(oracle.inv_helmholtz3(S0, S1, S2, D, u), want)
+    assert np.array_equal(oracle.inv_helmholtz3_bruteforce(S0, S1, S2, D, u), want)
+
+
+def test_inv_helmholtz3_special_cases_and_planted_mistakes():
+    g = rng(77)
+    nn = (3, 4, 2)
+    S0, S1, S2 = (g.standard_normal((n, n)) for n in nn)
+    D = g.uniform(0.1, 1.3, (2,) + nn)
+    u = g.uniform(-1, 1, (2,) + nn)
+    ref = ref_inv_helmholtz3_kron(S0, S1, S2, D, u)
+    # one shared matrix: the single-operator routine, bit for bit (same loops, same order)
+    n = 4
+    S = g.standard_normal((n, n))
+    Dc = g.uniform(0.1, 1.3, (2, n, n, n))
+    uc = g.uniform(-1, 1, (2, n, n, n))
+    assert np.array_equal(oracle.inv_helmholtz3(S, S, S, Dc, uc), oracle.inv_helmholtz(S, Dc, uc))
+    # identities on every axis: the pointwise product, bit for bit
+    I0, I1, I2 = (np.eye(k) for k in nn)
+    assert np.array_equal(oracle.inv_helmholtz3(I0, I1, I2, D, u), D * u)
+    # orthogonal operators, unit factor: the identity
+    Q0, Q1, Q2 = (np.linalg.qr(g.standard_normal((k, k)))[0] for k in nn)
+    assert relmax(oracle.inv_helmholtz3(Q0, Q1, Q2, np.ones_like(u), u), u) < 1e-13
+    # an identity on two axes leaves a one-axis operator: closed form with einsum
+    one = np.einsum("il,eljk->eijk", S0, D * np.einsum("li,eljk->eijk", S0, u))
+    assert relmax(oracle.inv_helmholtz3(S0, I1, I2, D, u), one) < 1e-13
+    # planted slips in the call must be seen by the library reference
+    assert relmax(oracle.inv_helmholtz3(S0.T, S1.T, S2.T, D, u), ref) > 1e-3      # transposes
+    assert relmax(oracle.inv_helmholtz3(S0, S1, S2, np.ones_like(D), u), ref) > 1e-3  # dropped D
+    nc = (3, 3, 3)
+    T0, T1, T2 = (g.standard_normal((3, 3)) for _ in range(3))
+    Dd = g.uniform(0.1, 1.3, (2,) + nc)
+    ud = g.uniform(-1, 1, (2,) + nc)
+    refc = ref_inv_helmholtz3_kron(T0, T1, T2, Dd, ud)
+    assert relmax(oracle.inv_helmholtz3(T2, T1, T0, Dd, ud), refc) > 1e-3         # direction order
+    assert relmax(oracle.inv_helmholtz3(T0, T2, T1, Dd, ud), refc) > 1e-3
+
+
+def test_rel_err_per_element_edge_cases():
+    ref = np.array([[1.0, 2.0, 2.0], [0.0, 0.0, 0.0], [3.0, 4.0, 0.0]])
+    v = ref.copy()
+    v[0, 0] = 1.0 + 3e-6
+    v[1, 0] = 1e-3                         # zero reference norm: guarded denominator
+    v[2, 1] = np.nan                       # any NaN in an element: infinite error
+    err = oracle.rel_err_per_element(v, ref)
+    assert abs(err[0] - 1e-6) < 1e-12
+    assert np.isfinite(err[1]) and err[1] > 1e290      # compared absolutely, against 1e-300
+    assert err[2] == np.inf
+    v[2, 1] = np.inf
+    assert oracle.rel_err_per_element(v, ref)[2] == np.inf
+    assert np.array_equal(oracle.rel_err_per_element(ref, ref), np.zeros(3))

@@ -22,6 +22,13 @@
  *    validates its arguments on the host, enqueues work on `stream` and returns.
  *    Buffers must stay valid until the stream has passed that work.  Inputs are
  *    only read; the output is fully overwritten.
+ *  - Work distribution: a launch in which a CTA gets more than one batch of
+ *    elements hands the batches out through a counter (16 bytes) taken from a fixed
+ *    ring of 4096 inside the library image and zeroed in stream order right before the
+ *    kernel (one cudaMemsetAsync on `stream`; it is captured with the kernel when
+ *    the stream is being captured).  A counter comes round again after 4096
+ *    launches; a kernel whose counter was touched by another launch while it ran
+ *    says so through ekl_tpo_device_error_flags (bit 1).
  *  - Errors: a status code is returned; nothing is thrown, aborted or trapped,
  *    and arguments that are accepted can never index out of bounds.  Validation
  *    happens before anything is enqueued:
@@ -81,13 +88,36 @@ ekl_tpo_status ekl_tpo_inv_helmholtz(const double* S, const double* D, const dou
  *
  * evaluated in exactly this order with IEEE operations, so the result equals
  * ekl_tpo_inv_helmholtz on the materialised D bit for bit.  Moves 16 n^3 + 8 bytes per
- * element instead of 24 n^3 and spends n^3 divisions.  fp64, 4 <= n <= 16 (other n:
+ * element instead of 24 n^3 and spends n^3 divisions.  fp64, 4 <= n <= 20 (other n:
  * EKL_TPO_ERR_UNSUPPORTED); even n needs a 16-byte aligned u (EKL_TPO_ERR_ALIGN otherwise).
  * v == u is allowed.
  */
 ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, const double* c,
                                             const double* u, double* v, int n, long long E,
                                             cudaStream_t stream);
+
+/*
+ * Inverse Helmholtz with one operator and one extent per direction.  The paper's operators
+ * carry a separate small matrix for every direction (Eq. 1 and the convective-flux listing
+ * of Sections 2.2 and 3 apply one matrix per axis); this is the inverse Helmholtz operator
+ * in that general form:
+ *
+ *     v[e] = (S0 (x) S1 (x) S2) . ( D[e] o ( (S0^T (x) S1^T (x) S2^T) . u[e] ) ),   e = 0..E-1
+ *
+ *   S0 [n0,n0]  S1 [n1,n1]  S2 [n2,n2]     S0 acts on the slowest in-element axis, S2 on the
+ *                                          contiguous one (Kronecker ordering of Eq. 1)
+ *   D,u,v [E,n0,n1,n2]                     D is multiplied pointwise
+ *
+ * fp64.  With S0 = S1 = S2 it equals ekl_tpo_inv_helmholtz.  v == u exactly (in place) is
+ * allowed; any other overlap of v with an input is rejected.  Extents are limited by shared
+ * memory (three matrices and two copies of an element).  The cubic shapes 8, 10, 12, 14, 16
+ * and the shapes (8,10,12), (12,10,8), (14,12,8), (8,8,16), (16,8,8), with a 16-byte aligned
+ * u, run on the FP64 tensor path; every other accepted shape runs on a general kernel with
+ * the same results to rounding.
+ */
+ekl_tpo_status ekl_tpo_inv_helmholtz3(const double* S0, const double* S1, const double* S2,
+                                      const double* D, const double* u, double* v,
+                                      int n0, int n1, int n2, long long E, cudaStream_t stream);
 
 /*
  * Forward rectangular tensor-product operator (the operator family of Eq. 1):
@@ -117,9 +147,9 @@ ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
  *   P   [3,3,E,nq,nq,nq]   fluxes, indexed [component][direction][element]...
  *   F   [3,E,nv,nv,nv]
  *
- * i.e. F[c,e,k,j,i] = sum_{l,m,n} ( D[i,l] I[j,m] I[k,n] P[c,0,e,n,m,l] + I[i,l] D[j,m] I[k,n]
- * P[c,1,e,n,m,l] + I[i,l] I[j,m] D[k,n] P[c,2,e,n,m,l] ) M[e,n,m,l]: the derivative acts on the
- * fastest axis for direction 0 and on the slowest for direction 2.  fp64.  F must not
+ * In each term the last Kronecker factor acts on the contiguous in-element axis, as everywhere
+ * in this header, so the differentiation matrix acts on the fastest axis for direction 0, on
+ * the middle one for direction 1 and on the slowest for direction 2.  fp64.  F must not
  * overlap any input.  (nq,nv) in {(4,4),(6,4),(6,6),(8,4),(8,6),(8,8),(10,8),(10,10),(12,8),
  * (12,10),(12,12),(14,12)} with 16-byte aligned M and P run on the FP64 tensor path; every
  * other combination that fits in shared memory (nq, nv <= 64 and about 2 max(nq,nv)^3 + nv^3
@@ -223,6 +253,10 @@ size_t ekl_tpo_host_workspace_bytes(long long in_elems_per_element, int n_inputs
  *    Issue them on one stream, or order them with events.
  *  - Work is enqueued on `stream` only (copy in, kernel, copy out, in that order); the
  *    result is in v once `stream` has reached the end of the call.  v == u is allowed.
+ *  - The status code is decided on the host when the work is enqueued; it cannot report
+ *    that a kernel's bounded wait gave up later on the device (v is then copied back
+ *    partly written).  A caller that wants to rule that out reads
+ *    ekl_tpo_device_error_flags() after synchronising.
  */
 #define EKL_TPO_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 ekl_tpo_status ekl_tpo_inv_helmholtz_host_static(const double* S, const double* D,
@@ -241,8 +275,10 @@ int ekl_tpo_last_cuda_error(void);
 /*
  * Device-side error flags since the last call of this function on the current device, and
  * clears them; -1 if the query itself failed.  Bit 0: a kernel's bounded wait on one of its
- * own bulk copies gave up (the kernel then stops early instead of hanging, and the output
- * of that launch is not valid).  Not expected in practice; meant for health checks.
+ * own bulk copies gave up (the kernel then stops early instead of hanging).  Bit 1: the
+ * work-distribution counter of a launch was written by something else while the kernel ran
+ * (see "Work distribution" above).  In both cases the output of that launch is not valid.
+ * Not expected in practice; meant for health checks.
  * SYNCHRONISES the device.  (Infrastructure: the paper has no counterpart.)
  */
 int ekl_tpo_device_error_flags(void);

@@ -102,7 +102,7 @@ ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, 
     if (n < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
     if (E == 0) return EKL_TPO_OK;
     if (!S || !lam || !c || !u || !v) return EKL_TPO_ERR_NULL;
-    if (n < 4 || n > 16) return EKL_TPO_ERR_UNSUPPORTED;
+    if (n < 4 || n > 20) return EKL_TPO_ERR_UNSUPPORTED;
     if (misaligned(S, 8) || misaligned(lam, 8) || misaligned(c, 8) || misaligned(u, 8) ||
         misaligned(v, 8) || (n % 2 == 0 && misaligned(u, 16)))
         return EKL_TPO_ERR_ALIGN;
@@ -115,6 +115,27 @@ ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, 
     cudaError_t err = cudaSuccess;
     if (!ekl::try_launch_ih_lambda_dmma(S, lam, c, u, v, n, E, stream, &err))
         return EKL_TPO_ERR_UNSUPPORTED;
+    return err == cudaSuccess ? EKL_TPO_OK : cuda_fail(err);
+}
+
+ekl_tpo_status ekl_tpo_inv_helmholtz3(const double* S0, const double* S1, const double* S2,
+                                      const double* D, const double* u, double* v, int n0, int n1,
+                                      int n2, long long E, cudaStream_t stream) {
+    if (n0 < 1 || n1 < 1 || n2 < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
+    if (E == 0) return EKL_TPO_OK;
+    if (!S0 || !S1 || !S2 || !D || !u || !v) return EKL_TPO_ERR_NULL;
+    if (!ekl::ih3_fits(n0, n1, n2, sizeof(double))) return EKL_TPO_ERR_UNSUPPORTED;
+    if (misaligned(S0, 8) || misaligned(S1, 8) || misaligned(S2, 8) || misaligned(D, 8) ||
+        misaligned(u, 8) || misaligned(v, 8))
+        return EKL_TPO_ERR_ALIGN;
+    const size_t field = (size_t)E * n0 * n1 * n2 * sizeof(double);
+    if (overlaps(v, field, S0, (size_t)n0 * n0 * sizeof(double)) ||
+        overlaps(v, field, S1, (size_t)n1 * n1 * sizeof(double)) ||
+        overlaps(v, field, S2, (size_t)n2 * n2 * sizeof(double)) || overlaps(v, field, D, field))
+        return EKL_TPO_ERR_OVERLAP;
+    if ((const void*)v != (const void*)u && overlaps(v, field, u, field))
+        return EKL_TPO_ERR_OVERLAP;
+    const cudaError_t err = ekl::launch_inv_helmholtz3(S0, S1, S2, D, u, v, n0, n1, n2, E, stream);
     return err == cudaSuccess ? EKL_TPO_OK : cuda_fail(err);
 }
 

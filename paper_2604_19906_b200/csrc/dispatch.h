@@ -21,6 +21,15 @@ inline int max_cubic_extent(size_t elem) {
     return n;
 }
 
+// The same for one operator and one extent per direction: three matrices + two element buffers.
+inline size_t generic_ih3_smem(int n0, int n1, int n2, size_t elem) {
+    return ((size_t)n0 * n0 + (size_t)n1 * n1 + (size_t)n2 * n2 + 2 * (size_t)n0 * n1 * n2) * elem;
+}
+inline bool ih3_fits(int n0, int n1, int n2, size_t elem) {
+    if ((double)n0 * n1 * n2 > 1.0e6 || n0 > 1000 || n1 > 1000 || n2 > 1000) return false;
+    return generic_ih3_smem(n0, n1, n2, elem) <= kMaxSmemBytes;
+}
+
 // Elements of one ping-pong buffer of the run-time-sized forward kernel.
 inline size_t generic_apply_buf(int n0, int n1, int n2, int m1, int m2) {
     size_t a = (size_t)n0 * n1 * n2, b = (size_t)n0 * n1 * m2, c = (size_t)n0 * m1 * m2;
@@ -62,14 +71,19 @@ cudaError_t launch_convection_generic(const double* Dvq, const double* Ivq, cons
                                       const double* P, double* F, int nq, int nv, long long E,
                                       cudaStream_t stream);
 
-// Bulk-copy timeout flag of the convective-flux kernels (see ekl_tpo_device_error_flags).
+// Device error flags of the convective-flux kernels and of the per-direction inverse
+// Helmholtz kernels (see ekl_tpo_device_error_flags).
 int convection_timeout_flag();
+int ih3_timeout_flag();
 
 // False when EKL_TPO_VARIANT=generic asks for the run-time-sized kernels only.
 bool tuned_kernels_allowed();
 
 // Number of SMs of the current device (cached per device).
 int sm_count();
+
+// A zeroed ticket counter (two 64-bit words) for one launch on `stream`; see launch.cu.
+cudaError_t next_ticket_counter(cudaStream_t stream, unsigned long long** out);
 
 // Tensor-path kernels (fp64 arithmetic; T is the type of the fields in memory).  Return false
 // if there is no instance for these extents or the pointers do not meet the alignment the
@@ -81,6 +95,10 @@ bool try_launch_ih_dmma(const T* S, const T* D, const T* u, T* v, int n, long lo
 bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double* cvec,
                                const double* u, double* v, int n, long long E, cudaStream_t stream,
                                cudaError_t* err);
+// One operator and one extent per direction (fp64).
+bool try_launch_ih3_dmma(const double* S0, const double* S1, const double* S2, const double* D,
+                         const double* u, double* v, int n0, int n1, int n2, long long E,
+                         cudaStream_t stream, cudaError_t* err);
 template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,
@@ -89,6 +107,10 @@ bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v,
 template <typename T>
 cudaError_t launch_inv_helmholtz(const T* S, const T* D, const T* u, T* v, int n, long long E,
                                  cudaStream_t stream);
+
+cudaError_t launch_inv_helmholtz3(const double* S0, const double* S1, const double* S2,
+                                  const double* D, const double* u, double* v, int n0, int n1,
+                                  int n2, long long E, cudaStream_t stream);
 
 template <typename T>
 cudaError_t launch_apply(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,

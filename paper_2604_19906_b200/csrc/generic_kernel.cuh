@@ -62,6 +62,42 @@ __global__ void inv_helmholtz_generic(const T* __restrict__ S, const T* __restri
     }
 }
 
+// v[e] = (S0(x)S1(x)S2)(D[e] o ((S0^T(x)S1^T(x)S2^T) u[e])): one operator and one extent per
+// direction, S0 on the slowest in-element axis.
+template <typename T>
+__global__ void inv_helmholtz3_generic(const T* __restrict__ S0, const T* __restrict__ S1,
+                                       const T* __restrict__ S2, const T* __restrict__ D,
+                                       const T* u, T* v, int n0, int n1, int n2, long long E) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T* s0 = reinterpret_cast<T*>(smem_raw);
+    T* s1 = s0 + n0 * n0;
+    T* s2 = s1 + n1 * n1;
+    const int n3 = n0 * n1 * n2;
+    T* b0 = s2 + n2 * n2;
+    T* b1 = b0 + n3;
+    for (int x = threadIdx.x; x < n0 * n0; x += blockDim.x) s0[x] = S0[x];
+    for (int x = threadIdx.x; x < n1 * n1; x += blockDim.x) s1[x] = S1[x];
+    for (int x = threadIdx.x; x < n2 * n2; x += blockDim.x) s2[x] = S2[x];
+    for (long long e = blockIdx.x; e < E; e += gridDim.x) {
+        const T* ue = u + e * n3;
+        const T* De = D + e * n3;
+        __syncthreads();
+        for (int x = threadIdx.x; x < n3; x += blockDim.x) b0[x] = ue[x];
+        __syncthreads();
+        contract_axis<T, T>(b0, b1, s2, 1, n2, n0, n1, n2, 2, n2, nullptr);   // S2^T, fast axis
+        __syncthreads();
+        contract_axis<T, T>(b1, b0, s1, 1, n1, n0, n1, n2, 1, n1, nullptr);
+        __syncthreads();
+        contract_axis<T, T>(b0, b1, s0, 1, n0, n0, n1, n2, 0, n0, De);        // ... and times D[e]
+        __syncthreads();
+        contract_axis<T, T>(b1, b0, s2, n2, 1, n0, n1, n2, 2, n2, nullptr);   // S2, fast axis
+        __syncthreads();
+        contract_axis<T, T>(b0, b1, s1, n1, 1, n0, n1, n2, 1, n1, nullptr);
+        __syncthreads();
+        contract_axis<T, T>(b1, v + e * n3, s0, n0, 1, n0, n1, n2, 0, n0, nullptr);
+    }
+}
+
 // v[e] = (A(x)B(x)C) u[e], contraction order C, B, A.
 template <typename T>
 __global__ void apply_generic(const T* __restrict__ A, const T* __restrict__ B,

@@ -30,12 +30,13 @@
 namespace ekl {
 namespace dmma {
 
-// Set by a kernel whose bounded wait on a bulk copy gave up (not expected in practice).  Every
-// translation unit that includes this header has its own copy and reads it with
-// take_timeout_flag().
+// Bit 0: a kernel's bounded wait on a bulk copy gave up.  Bit 1: the ticket counter of a launch
+// did not end at the value its own draws add up to, i.e. something else wrote to it while the
+// kernel ran.  Neither is expected in practice.  Every translation unit that includes this
+// header has its own copy and reads it with take_timeout_flag().
 static __device__ int g_bulk_wait_timeout = 0;
 
-// Host: this translation unit's flag (1 = a wait gave up, -1 = the query failed), cleared.
+// Host: this translation unit's flags (-1 = the query failed), cleared.
 static inline int take_timeout_flag() {
     int flag = 0;
     if (cudaMemcpyFromSymbol(&flag, g_bulk_wait_timeout, sizeof(int)) != cudaSuccess) return -1;
@@ -43,8 +44,70 @@ static inline int take_timeout_flag() {
         const int zero = 0;
         cudaMemcpyToSymbol(g_bulk_wait_timeout, &zero, sizeof(int));
     }
-    return flag ? 1 : 0;
+    return flag & 3;
 }
+
+// Hands the batches of a launch to its CTAs.  Every CTA starts on batch blockIdx.x.  With a
+// ticket counter (two 64-bit words in global memory, zeroed in stream order before the launch)
+// the later batches go to whichever CTA asks first: co-resident CTAs do not get equal shares of
+// an SM, and a fixed round-robin share makes the launch wait for the slowest of them.  A CTA
+// always knows its next batch one iteration ahead (it prefetches that batch), so a ticket is
+// drawn at the top of an iteration and used two iterations later.  Without a counter
+// (nullptr) the batches are dealt round-robin.
+struct BatchQueue {
+    unsigned long long* ticket;
+    long long* shared_next;       // one value in shared memory
+    long long batch, next;
+    unsigned long long drawn;
+
+    // All threads; the caller synchronises the CTA before started().
+    __device__ __forceinline__ void start(unsigned long long* t, long long* sh) {
+        ticket = t;
+        shared_next = sh;
+        batch = blockIdx.x;
+        next = batch + gridDim.x;
+        drawn = 0;
+        if (ticket && threadIdx.x == 0) *sh = (long long)gridDim.x + (long long)atomicAdd(ticket, 1ull);
+    }
+    __device__ __forceinline__ void started() {
+        if (ticket) next = *shared_next;
+    }
+    // Top of an iteration: ask for the batch after next.
+    __device__ __forceinline__ void draw() {
+        if (ticket && threadIdx.x == 0) drawn = atomicAdd(ticket, 1ull);
+    }
+    // Before a CTA barrier at or after the end of the iteration.
+    __device__ __forceinline__ void publish() {
+        if (ticket && threadIdx.x == 0) *shared_next = (long long)gridDim.x + (long long)drawn;
+    }
+    // After that barrier.
+    __device__ __forceinline__ void advance() {
+        batch = next;
+        next = ticket ? *shared_next : next + gridDim.x;
+    }
+    // For a loop whose iterations end without a barrier: advance_batch() after publish(),
+    // refresh() after the first barrier of the following iteration.
+    __device__ __forceinline__ void advance_batch() {
+        batch = next;
+        if (!ticket) next += gridDim.x;
+    }
+    __device__ __forceinline__ void refresh() {
+        if (ticket) next = *shared_next;
+    }
+    // End of the kernel: the CTA that leaves last checks that the counter holds exactly the
+    // draws of this launch (one per CTA at the start, one per batch).
+    __device__ __forceinline__ void finish(long long n_batches) {
+        if (ticket && threadIdx.x == 0) {
+            __threadfence();
+            const unsigned long long gone = atomicAdd(ticket + 1, 1ull);
+            if (gone == gridDim.x - 1) {
+                const unsigned long long draws = atomicAdd(ticket, 0ull);
+                if (draws != (unsigned long long)gridDim.x + (unsigned long long)n_batches)
+                    atomicOr(&g_bulk_wait_timeout, 2);
+            }
+        }
+    }
+};
 
 __device__ __forceinline__ void mma_f64(double& c0, double& c1, double a, double b) {
     asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
@@ -112,7 +175,7 @@ __device__ __forceinline__ void fence_async_proxy() {
 // wait gave up; the decision is the same for every thread.
 __device__ __forceinline__ bool wait_bulk(uint64_t* bar, unsigned parity) {
     if (__syncthreads_or(mbar_wait(bar, parity) ? 0 : 1)) {
-        if (threadIdx.x == 0) g_bulk_wait_timeout = 1;
+        if (threadIdx.x == 0) atomicOr(&g_bulk_wait_timeout, 1);
         mbar_wait(bar, parity);
         return false;
     }
@@ -436,7 +499,7 @@ template <int N, typename T, bool LAMBDA = false>
 __global__ void __launch_bounds__(IhCfg<N, T>::kThreads, IhCfg<N, T>::kCtasPerSm)
 inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
                    const double* __restrict__ lam, const double* __restrict__ cvec, const T* u,
-                   T* v, long long E) {
+                   T* v, long long E, unsigned long long* tickets) {
     using C = IhCfg<N, T>;
     constexpr bool kBulk = C::kBulk && sizeof(T) == sizeof(double);
     using First = typename C::First;
@@ -462,15 +525,19 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
     load_op<Mid, T>(opb, S, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    __shared__ long long shared_next;
+    BatchQueue q;
+    q.start(tickets, &shared_next);
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
+    q.started();
 
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
-    long long batch = blockIdx.x;
-    if (batch < n_batches) {
+    if (q.batch < n_batches) {
+        const long long batch = q.batch;
         if (kStaged)
             stage_floats(staging, reinterpret_cast<const float*>(u) + batch * C::kBe * kN3,
                          batch_count(batch) * kN3);
@@ -483,7 +550,9 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
                 bar);
     }
     unsigned parity = 0;
-    for (; batch < n_batches; batch += gridDim.x) {
+    while (q.batch < n_batches) {
+        q.draw();
+        const long long batch = q.batch, next = q.next;
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
         const int valid = cnt * kN2;
@@ -496,7 +565,6 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
             fac.Db = D + e0 * kN3;
         }
         const NoFactor none;
-        const long long next = batch + gridDim.x;
         if (threadIdx.x == 0 && next < n_batches) {
             const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(T));
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
@@ -545,8 +613,138 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
             }
         }
         run_stage<Last, 2, T, NoFactor, FD>(bufB, nullptr, v + e0 * kN3, opb, dfac, none, valid, warp, lane);
+        q.publish();
         __syncthreads();
+        q.advance();
     }
+    q.finish(n_batches);
+}
+
+// ------------------------------------------------------------------ inverse Helmholtz, one
+// operator and one extent per direction
+
+template <int N0, int N1, int N2>
+struct Ih3Cfg {
+    static constexpr int cmax(int a, int b) { return a > b ? a : b; }
+    // u as it lands: [n0][n1*n2] with padded planes
+    static constexpr int kPS0 = pad_plane(N1 * N2), kES0 = N0 * kPS0;
+    // after contracting axis 0: [n1][n2][o0]; after axis 1: [n2][o0][o1]; after axis 2 the
+    // natural order [o0][o1][o2] again (kept in shared memory between the two halves)
+    static constexpr int kRS1 = pad_row(N0), kPS1 = pad_plane(N2 * kRS1), kES1 = N1 * kPS1;
+    static constexpr int kRS2 = pad_row(N1), kPS2 = pad_plane(N0 * kRS2), kES2 = N2 * kPS2;
+    static constexpr int kRS3 = pad_row(N2), kPS3 = pad_plane(N1 * kRS3), kES3 = N0 * kPS3;
+    static constexpr int kElemBuf = cmax(cmax(kES0, kES1), cmax(kES2, kES3));
+    // two elements per batch unless that leaves room for one CTA per SM only
+    static constexpr int kBe = (4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1;
+    static constexpr int kMaxTiles =
+        (kBe * cmax(cmax(N1 * N2, N2 * N0), N0 * N1) + 7) / 8;
+    static constexpr int kWarps = (kMaxTiles > 36) ? 8 : 4;
+    using F1 = Stage<N0, N0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
+    using F2 = Stage<N1, N1, N2, N0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
+    using F3 = Stage<N2, N2, N0, N1, kBe, kWarps, kRS2, kPS2, kES2, kRS3, kPS3, kES3>;
+    using B1 = Stage<N0, N0, N1, N2, kBe, kWarps, kRS3, kPS3, kES3, kRS1, kPS1, kES1>;
+    using B3 = Stage<N2, N2, N0, N1, kBe, kWarps, kRS2, kPS2, kES2, N2, N1 * N2, N0 * N1 * N2>;
+    static constexpr int kThreads = 32 * kWarps;
+    static constexpr int kBufElems = kBe * kElemBuf;
+    static constexpr size_t kSmemBytes = 2 * (size_t)kBufElems * sizeof(double) + 16;
+    static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
+    static constexpr int kByWarps = 20 / kWarps;
+    static constexpr int kCtasPerSm =
+        (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
+    static_assert(N0 % 2 == 0 && N1 % 2 == 0 && N2 % 2 == 0 && N0 >= 4 && N1 >= 4 && N2 >= 4,
+                  "even extents from 4 (bulk copies work in 16-byte units)");
+};
+
+// v[e] = (S0(x)S1(x)S2)(D[e] o ((S0^T(x)S1^T(x)S2^T) u[e])), fp64, u 16-byte aligned.  The
+// operator fragments of a stage are fetched while the stage before it runs, so that two sets
+// are live at a time whatever the number of distinct matrices.
+template <int N0, int N1, int N2>
+__global__ void __launch_bounds__(Ih3Cfg<N0, N1, N2>::kThreads, Ih3Cfg<N0, N1, N2>::kCtasPerSm)
+inv_helmholtz3_dmma(const double* __restrict__ S0, const double* __restrict__ S1,
+                    const double* __restrict__ S2, const double* __restrict__ D, const double* u,
+                    double* v, long long E, unsigned long long* tickets) {
+    using C = Ih3Cfg<N0, N1, N2>;
+    using T = double;
+    using F1 = typename C::F1;
+    using F2 = typename C::F2;
+    using F3 = typename C::F3;
+    using B1 = typename C::B1;
+    using B3 = typename C::B3;
+    constexpr int kN3 = N0 * N1 * N2;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    double* bufA = reinterpret_cast<double*>(smem_raw);
+    double* bufB = bufA + C::kBufElems;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(bufB + C::kBufElems);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = ((threadIdx.x >> 5) + blockIdx.x) % C::kWarps;
+
+    const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    __shared__ long long shared_next;
+    BatchQueue q;
+    q.start(tickets, &shared_next);
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    __syncthreads();
+    q.started();
+    auto batch_count = [&](long long b) {
+        const long long e0 = b * C::kBe;
+        return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
+    };
+    if (q.batch < n_batches && threadIdx.x == 0)
+        load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufA, u + q.batch * C::kBe * kN3,
+                                                     batch_count(q.batch), bar);
+    OpFrag<F1> f1;
+    OpFrag<F2> f2;
+    OpFrag<F3> f3;
+    load_op<F1, T>(f1, S0, false, lane);
+    unsigned parity = 0;
+    double dfac[1][F3::kMTiles][2], none1[1][F1::kMTiles][2], none2[1][F2::kMTiles][2];
+    const NoFactor none;
+    while (q.batch < n_batches) {
+        q.draw();
+        const long long batch = q.batch, next = q.next;
+        const long long e0 = batch * C::kBe;
+        const int cnt = batch_count(batch);
+        FieldFactor<T> fac;
+        fac.Db = D + e0 * kN3;
+        if (threadIdx.x == 0 && next < n_batches) {
+            const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(T));
+            bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
+            bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
+        }
+        if (!wait_bulk(bar, parity)) break;
+        parity ^= 1u;
+        // forward: S0^T on the slowest axis, then S1^T, then S2^T
+        load_op<F2, T>(f2, S1, false, lane);
+        run_stage<F1, 0, T, NoFactor, 1>(bufA, bufB, nullptr, f1, none1, none, cnt * F1::kP, warp, lane);
+        __syncthreads();
+        load_op<F3, T>(f3, S2, false, lane);
+        fac.template load<F3>(dfac[0], cnt * F3::kP, warp, 0, lane);
+        run_stage<F2, 0, T, NoFactor, 1>(bufB, bufA, nullptr, f2, none2, none, cnt * F2::kP, warp, lane);
+        __syncthreads();
+        load_op<F1, T>(f1, S0, true, lane);
+        run_stage<F3, 1, T, FieldFactor<T>, 1>(bufA, bufB, nullptr, f3, dfac, fac, cnt * F3::kP, warp, lane);
+        __syncthreads();
+        // backward: S0, S1, S2 themselves
+        load_op<F2, T>(f2, S1, true, lane);
+        run_stage<B1, 0, T, NoFactor, 1>(bufB, bufA, nullptr, f1, none1, none, cnt * B1::kP, warp, lane);
+        __syncthreads();
+        load_op<F3, T>(f3, S2, true, lane);
+        run_stage<F2, 0, T, NoFactor, 1>(bufA, bufB, nullptr, f2, none2, none, cnt * F2::kP, warp, lane);
+        __syncthreads();
+        // bufA is free: bring in the next batch while the last stage streams v out
+        if (next < n_batches && threadIdx.x == 0) {
+            fence_async_proxy();
+            load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
+                                                         batch_count(next), bar);
+        }
+        load_op<F1, T>(f1, S0, false, lane);
+        run_stage<B3, 2, T, NoFactor, 1>(bufB, nullptr, v + e0 * kN3, f3, dfac, none, cnt * B3::kP, warp, lane);
+        q.publish();
+        __syncthreads();
+        q.advance();
+    }
+    q.finish(n_batches);
 }
 
 // ------------------------------------------------------------------ forward rectangular operator
@@ -583,7 +781,7 @@ template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
 __global__ void __launch_bounds__(ApplyCfg<N0, N1, N2, M0, M1, M2>::kThreads,
                                   ApplyCfg<N0, N1, N2, M0, M1, M2>::kCtasPerSm)
 apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict__ Cm,
-           const T* __restrict__ u, T* __restrict__ v, long long E) {
+           const T* __restrict__ u, T* __restrict__ v, long long E, unsigned long long* tickets) {
     using C = ApplyCfg<N0, N1, N2, M0, M1, M2>;
     constexpr bool kBulk = sizeof(T) == sizeof(double);
     using S1 = typename C::S1;
@@ -607,13 +805,15 @@ apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict
     load_op<S3, T>(opC, Cm, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    __shared__ long long shared_next;
+    BatchQueue q;
+    q.start(tickets, &shared_next);
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
-    long long batch = blockIdx.x;
     auto fetch = [&](long long b) {
         if (!kBulk) {
             copy_elements<N0, N1 * N2, C::kPS0, C::kES0, T>(bufU, u + b * C::kBe * S1::kIn,
@@ -624,19 +824,22 @@ apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict
                 bufU, reinterpret_cast<const double*>(u) + b * C::kBe * S1::kIn, batch_count(b), bar);
         }
     };
-    if (batch < n_batches) fetch(batch);
+    if (q.batch < n_batches) fetch(q.batch);
     unsigned parity = 0;
     double none1[1][S1::kMTiles][2], none2[1][S2::kMTiles][2], none3[1][S3::kMTiles][2];
-    for (; batch < n_batches; batch += gridDim.x) {
+    while (q.batch < n_batches) {
+        q.draw();
+        const long long batch = q.batch;
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
-        const long long next = batch + gridDim.x;
         if (kBulk) {
             if (!wait_bulk(bar, parity)) break;
             parity ^= 1u;
         } else {
             wait_copies();
         }
+        q.refresh();
+        const long long next = q.next;
         run_stage<S1, 0, T>(bufU, bufB, nullptr, opA, none1, NoFactor(), cnt * S1::kP, warp, lane);
         __syncthreads();
         // the landing buffer is free: bring in the next batch under the remaining two stages
@@ -645,8 +848,12 @@ apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict
         __syncthreads();
         run_stage<S3, 2, T>(bufA, nullptr, v + e0 * S3::kOut, opC, none3, NoFactor(), cnt * S3::kP,
                             warp, lane);
-        // the next batch's first stage writes bufB, which this batch no longer reads
+        // the next batch's first stage writes bufB, which this batch no longer reads; the
+        // barrier in the next iteration's wait orders the ticket handed over here
+        q.publish();
+        q.advance_batch();
     }
+    q.finish(n_batches);
 }
 
 }  // namespace dmma

@@ -2,6 +2,7 @@
 #include <cstdint>
 
 #include "dispatch.h"
+#include "launch_util.h"
 #include "tpo_dmma.cuh"
 #include "tpo_tf32.cuh"
 #include "tpo_umma.cuh"
@@ -12,34 +13,11 @@
 namespace ekl {
 namespace {
 
-// Opts the kernel into its dynamic shared memory and asks how many CTAs fit on an SM; done
-// once per device and kernel (the answer is kept), so that repeated calls cost one launch.
-// Racing first calls compute the same value.
-// `cached` is the caller's per-kernel table (kernels of different shapes can share a
-// function-pointer type, so the table cannot live here).
-template <typename Kernel>
-cudaError_t ctas_per_sm(Kernel kernel, int threads, size_t smem, int (&cached)[64], int* per_sm) {
-    int dev = 0;
-    cudaError_t err = cudaGetDevice(&dev);
-    if (err != cudaSuccess) return err;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (cached[dev] == 0) {
-        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return err;
-        int n = 1;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem);
-        if (err != cudaSuccess) return err;
-        cached[dev] = n < 1 ? 1 : n;
-    }
-    *per_sm = cached[dev];
-    return cudaSuccess;
-}
-
 template <int N, typename T, bool LAMBDA>
 cudaError_t launch_ih(const T* S, const T* D, const double* lam, const double* cvec, const T* u, T* v,
                       long long E, cudaStream_t stream) {
     using C = dmma::IhCfg<N, T>;
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int per_sm = 1;
     cudaError_t err = ctas_per_sm(dmma::inv_helmholtz_dmma<N, T, LAMBDA>, C::kThreads,
                                   C::kSmemBytes, cached, &per_sm);
@@ -47,8 +25,11 @@ cudaError_t launch_ih(const T* S, const T* D, const double* lam, const double* c
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
+    unsigned long long* tickets = nullptr;
+    err = tickets_for(batches, grid, stream, &tickets);
+    if (err != cudaSuccess) return err;
     dmma::inv_helmholtz_dmma<N, T, LAMBDA>
-        <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, lam, cvec, u, v, E);
+        <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, lam, cvec, u, v, E, tickets);
     return cudaGetLastError();
 }
 
@@ -57,7 +38,7 @@ template <int N>
 cudaError_t launch_ih_tf32(const float* S, const float* D, const float* u, float* v, long long E,
                            cudaStream_t stream) {
     using C = tf32::IhCfg32<N>;
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int per_sm = 1;
     cudaError_t err = ctas_per_sm(tf32::inv_helmholtz_tf32<N>, C::kThreads, C::kSmemBytes, cached,
                                   &per_sm);
@@ -65,7 +46,11 @@ cudaError_t launch_ih_tf32(const float* S, const float* D, const float* u, float
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
-    tf32::inv_helmholtz_tf32<N><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E);
+    unsigned long long* tickets = nullptr;
+    err = tickets_for(batches, grid, stream, &tickets);
+    if (err != cudaSuccess) return err;
+    tf32::inv_helmholtz_tf32<N>
+        <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E, tickets);
     return cudaGetLastError();
 }
 
@@ -139,14 +124,17 @@ cudaError_t launch_ap_tf32(const float* A, const float* B, const float* Cm, cons
                            long long E, cudaStream_t stream) {
     using C = tf32::ApplyCfg32<N, N, N, M, M, M>;
     auto kernel = tf32::apply_tf32<N, N, N, M, M, M>;
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int per_sm = 1;
     cudaError_t err = ctas_per_sm(kernel, C::kThreads, C::kSmemBytes, cached, &per_sm);
     if (err != cudaSuccess) return err;
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
-    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E);
+    unsigned long long* tickets = nullptr;
+    err = tickets_for(batches, grid, stream, &tickets);
+    if (err != cudaSuccess) return err;
+    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
     return cudaGetLastError();
 }
 
@@ -184,14 +172,17 @@ cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, lon
                       cudaStream_t stream) {
     using C = dmma::ApplyCfg<N0, N1, N2, M0, M1, M2>;
     auto kernel = dmma::apply_dmma<N0, N1, N2, M0, M1, M2, T>;
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];
     int per_sm = 1;
     cudaError_t err = ctas_per_sm(kernel, C::kThreads, C::kSmemBytes, cached, &per_sm);
     if (err != cudaSuccess) return err;
     const long long batches = (E + C::kBe - 1) / C::kBe;
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
-    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E);
+    unsigned long long* tickets = nullptr;
+    err = tickets_for(batches, grid, stream, &tickets);
+    if (err != cudaSuccess) return err;
+    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
     return cudaGetLastError();
 }
 
@@ -268,6 +259,10 @@ bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double*
         EKL_LAMBDA_CASE(14)
         EKL_LAMBDA_CASE(15)
         EKL_LAMBDA_CASE(16)
+        EKL_LAMBDA_CASE(17)
+        EKL_LAMBDA_CASE(18)
+        EKL_LAMBDA_CASE(19)
+        EKL_LAMBDA_CASE(20)
 #undef EKL_LAMBDA_CASE
         default: return false;
     }
@@ -307,11 +302,13 @@ template bool try_launch_apply_dmma<float>(const float*, const float*, const flo
 }  // namespace ekl
 
 // Reads (and clears) the flags device code raises when something that should never happen
-// did: bit 0 = a bounded wait on a bulk copy gave up, so the results of that launch are
-// not valid.  Synchronises the device.
+// did: bit 0 = a bounded wait on a bulk copy gave up, bit 1 = a launch's ticket counter was
+// written by something else while it ran; either way the results of that launch are not
+// valid.  Synchronises the device.
 extern "C" int ekl_tpo_device_error_flags(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-    const int a = ekl::dmma::take_timeout_flag(), b = ekl::convection_timeout_flag();
-    if (a < 0 || b < 0) return -1;
-    return (a | b) ? 1 : 0;
+    const int a = ekl::dmma::take_timeout_flag(), b = ekl::convection_timeout_flag(),
+              c = ekl::ih3_timeout_flag();
+    if (a < 0 || b < 0 || c < 0) return -1;
+    return a | b | c;
 }

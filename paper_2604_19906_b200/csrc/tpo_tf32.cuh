@@ -186,9 +186,8 @@ __device__ __forceinline__ void load_elements32(float* dst, const float* src, in
     }
 }
 
-#ifndef EKL_TF32_MAX_WARPS
-#define EKL_TF32_MAX_WARPS 24
-#endif
+// at most this many warps of these kernels share an SM (measured best)
+constexpr int kMaxWarpsPerSm = 24;
 
 template <int N>
 struct IhCfg32 {
@@ -211,7 +210,7 @@ struct IhCfg32 {
     static constexpr int kBufElems = kBe * kElemBuf;
     static constexpr size_t kSmemBytes = 2 * (size_t)kBufElems * sizeof(float) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
-    static constexpr int kByWarps = EKL_TF32_MAX_WARPS / kWarps;
+    static constexpr int kByWarps = kMaxWarpsPerSm / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
     static constexpr int kFactorDepth = (Mid::kTilesPerWarp >= 6) ? 4 : 2;
@@ -221,7 +220,7 @@ struct IhCfg32 {
 template <int N>
 __global__ void __launch_bounds__(IhCfg32<N>::kThreads, IhCfg32<N>::kCtasPerSm)
 inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, const float* u, float* v,
-                   long long E) {
+                   long long E, unsigned long long* tickets) {
     using C = IhCfg32<N>;
     using First = typename C::First;
     using Mid = typename C::Mid;
@@ -242,23 +241,27 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
     load_op32<Mid>(opb, S, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    __shared__ long long shared_next;
+    dmma::BatchQueue q;
+    q.start(tickets, &shared_next);
     if (threadIdx.x == 0) dmma::mbar_init(bar, 1);
     __syncthreads();
+    q.started();
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
-    long long batch = blockIdx.x;
-    if (batch < n_batches && threadIdx.x == 0)
-        load_elements32<N, kN2, C::kPS0, C::kES0>(bufA, u + batch * C::kBe * kN3, batch_count(batch),
-                                                  bar);
+    if (q.batch < n_batches && threadIdx.x == 0)
+        load_elements32<N, kN2, C::kPS0, C::kES0>(bufA, u + q.batch * C::kBe * kN3,
+                                                  batch_count(q.batch), bar);
     unsigned parity = 0;
-    for (; batch < n_batches; batch += gridDim.x) {
+    while (q.batch < n_batches) {
+        q.draw();
+        const long long batch = q.batch, next = q.next;
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
         const int valid = cnt * kN2;
         const float* Db = D + e0 * kN3;
-        const long long next = batch + gridDim.x;
         if (threadIdx.x == 0 && next < n_batches) {
             const unsigned nbytes = (unsigned)(batch_count(next) * kN3 * sizeof(float));
             dmma::bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
@@ -288,8 +291,11 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
                                                       batch_count(next), bar);
         }
         run_stage32<Last, 2, FD>(bufB, nullptr, v + e0 * kN3, opb, dfac, Db, valid, warp, lane);
+        q.publish();
         __syncthreads();
+        q.advance();
     }
+    q.finish(n_batches);
 }
 
 // ------------------------------------------------------------------ forward rectangular operator
@@ -308,10 +314,8 @@ struct ApplyCfg32 {
     static constexpr int kMaxTiles =
         kBe * (N1 * N2 > N2 * M0 ? (N1 * N2 > M0 * M1 ? N1 * N2 : M0 * M1)
                                  : (N2 * M0 > M0 * M1 ? N2 * M0 : M0 * M1)) / 8;
-#ifndef EKL_TF32_APPLY_TILES_FOR_8
-#define EKL_TF32_APPLY_TILES_FOR_8 48
-#endif
-    static constexpr int kWarps = (kMaxTiles > EKL_TF32_APPLY_TILES_FOR_8) ? 8 : 4;
+    // 4-warp CTAs up to 48 tiles per stage (measured), 8 beyond
+    static constexpr int kWarps = (kMaxTiles > 48) ? 8 : 4;
     using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;
     using S2 = Stage<N1, M1, N2, M0, kBe, kWarps, kRS1, kPS1, kES1, kRS2, kPS2, kES2>;
     using S3 = Stage<N2, M2, M0, M1, kBe, kWarps, kRS2, kPS2, kES2, M2, M1 * M2, M0 * M1 * M2>;
@@ -319,10 +323,7 @@ struct ApplyCfg32 {
     static constexpr int kU = kBe * kES0, kB = kBe * kES1, kA = kBe * kES2;
     static constexpr size_t kSmemBytes = (size_t)(kU + kB + kA) * sizeof(float) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
-#ifndef EKL_TF32_APPLY_MAX_WARPS
-#define EKL_TF32_APPLY_MAX_WARPS EKL_TF32_MAX_WARPS
-#endif
-    static constexpr int kByWarps = EKL_TF32_APPLY_MAX_WARPS / kWarps;
+    static constexpr int kByWarps = kMaxWarpsPerSm / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
     static_assert((N1 * N2) % 4 == 0, "planes must be a whole number of 16-byte units");
@@ -334,7 +335,8 @@ template <int N0, int N1, int N2, int M0, int M1, int M2>
 __global__ void __launch_bounds__(ApplyCfg32<N0, N1, N2, M0, M1, M2>::kThreads,
                                   ApplyCfg32<N0, N1, N2, M0, M1, M2>::kCtasPerSm)
 apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float* __restrict__ Cm,
-           const float* __restrict__ u, float* __restrict__ v, long long E) {
+           const float* __restrict__ u, float* __restrict__ v, long long E,
+           unsigned long long* tickets) {
     using C = ApplyCfg32<N0, N1, N2, M0, M1, M2>;
     using S1 = typename C::S1;
     using S2 = typename C::S2;
@@ -357,6 +359,9 @@ apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float
     load_op32<S3>(opC, Cm, true, lane);
 
     const long long n_batches = (E + C::kBe - 1) / C::kBe;
+    __shared__ long long shared_next;
+    dmma::BatchQueue q;
+    q.start(tickets, &shared_next);
     if (threadIdx.x == 0) dmma::mbar_init(bar, 1);
     __syncthreads();
     auto batch_count = [&](long long b) {
@@ -370,16 +375,18 @@ apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float
                                                            batch_count(b), bar);
         }
     };
-    long long batch = blockIdx.x;
-    if (batch < n_batches) fetch(batch);
+    if (q.batch < n_batches) fetch(q.batch);
     unsigned parity = 0;
     float none[1][4];
-    for (; batch < n_batches; batch += gridDim.x) {
+    while (q.batch < n_batches) {
+        q.draw();
+        const long long batch = q.batch;
         const long long e0 = batch * C::kBe;
         const int cnt = batch_count(batch);
-        const long long next = batch + gridDim.x;
         if (!dmma::wait_bulk(bar, parity)) break;
         parity ^= 1u;
+        q.refresh();
+        const long long next = q.next;
         run_stage32<S1, 0, 1>(bufU, bufB, nullptr, opA, none, nullptr, cnt * S1::kP, warp, lane);
         __syncthreads();
         // the landing buffer is free: bring in the next batch under the remaining two stages
@@ -388,8 +395,12 @@ apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float
         __syncthreads();
         run_stage32<S3, 2, 1>(bufA, nullptr, v + e0 * S3::kOut, opC, none, nullptr, cnt * S3::kP, warp,
                               lane);
-        // the next batch's first stage writes bufB, which this batch no longer reads
+        // the next batch's first stage writes bufB, which this batch no longer reads; the
+        // barrier in the next iteration's wait orders the ticket handed over here
+        q.publish();
+        q.advance_batch();
     }
+    q.finish(n_batches);
 }
 
 }  // namespace tf32

@@ -137,9 +137,35 @@ def ekl_tpo_apply_f32(A, B, C, u, out=None):
     return _apply("ekl_tpo_apply_f32", torch.float32, A, B, C, u, out)
 
 
+def ekl_tpo_inv_helmholtz3(S0, S1, S2, D, u, out=None):
+    """``v[e] = (S0⊗S1⊗S2)·(D[e] ∘ ((S0ᵀ⊗S1ᵀ⊗S2ᵀ)·u[e]))``: one operator and one extent per
+    direction, fp64, on the current stream.  ``out`` may be ``u`` itself (in place)."""
+    lib = library()
+    fn = lib.ekl_tpo_inv_helmholtz3
+    fn.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int] * 3 + [ctypes.c_longlong, ctypes.c_void_p]
+    fn.restype = ctypes.c_int
+    if u.dim() != 4 or any(S.dim() != 2 or S.shape[0] != S.shape[1] for S in (S0, S1, S2)):
+        raise ValueError("S0, S1, S2 must be square matrices and u [E,n0,n1,n2]")
+    nn = (S0.shape[0], S1.shape[0], S2.shape[0])
+    if tuple(u.shape[1:]) != nn or D.shape != u.shape:
+        raise ValueError("D and u must be [E,n0,n1,n2] with n_d the order of S_d")
+    dev = u.device
+    if out is None:
+        out = torch.empty_like(u)
+    elif out.shape != u.shape:
+        raise ValueError("out must have the shape of u")
+    ptrs = [_dev_ptr(t, nm, torch.float64, dev)
+            for t, nm in ((S0, "S0"), (S1, "S1"), (S2, "S2"), (D, "D"), (u, "u"), (out, "out"))]
+    with torch.cuda.device(dev):
+        st = fn(*ptrs, *nn, u.shape[0], _stream(dev))
+    if st:
+        raise EklTpoError(st, "ekl_tpo_inv_helmholtz3")
+    return out
+
+
 def ekl_tpo_inv_helmholtz_lambda(S, lam, c, u, out=None):
     """Inverse Helmholtz with ``D[e,i,j,k] = 1/(((lam[i]+lam[j])+lam[k])+c[e])`` formed on the
-    fly (fp64, 4 <= n <= 16); bit-identical to :func:`ekl_tpo_inv_helmholtz` on that D."""
+    fly (fp64, 4 <= n <= 20); bit-identical to :func:`ekl_tpo_inv_helmholtz` on that D."""
     lib = library()
     fn = lib.ekl_tpo_inv_helmholtz_lambda
     fn.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p]

@@ -14,9 +14,11 @@ def env():
     return {"torch": torch, "oracle": oracle, "ops": ops, "dev": torch.device("cuda:0")}
 
 
-@pytest.mark.parametrize("n", list(range(4, 17)))
+@pytest.mark.parametrize("n", list(range(4, 21)))
 @pytest.mark.parametrize("E", [1, 3, 130, 1501])
 def test_lambda_variant_matches_oracle_and_field_variant(env, n, E):
+    if n > 16 and E > 130:
+        E = 301
     torch, ops = env["torch"], env["ops"]
     g = np.random.Generator(np.random.PCG64(31 * n + E))
     S, _ = np.linalg.qr(g.standard_normal((n, n)))
@@ -40,7 +42,7 @@ def test_lambda_variant_matches_oracle_and_field_variant(env, n, E):
 def test_lambda_variant_refuses_what_it_cannot_do(env):
     torch, ops = env["torch"], env["ops"]
     dev = env["dev"]
-    for n in (3, 17):
+    for n in (3, 21):
         S = torch.eye(n, dtype=torch.float64, device=dev)
         lam = torch.ones(n, dtype=torch.float64, device=dev)
         c = torch.ones(2, dtype=torch.float64, device=dev)

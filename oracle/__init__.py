@@ -20,7 +20,7 @@ Operators (row-major arrays, element index slowest, see ``tpo_oracle.c``):
   operator family of Eq. 1.
 * ``convection(Dvq, Ivq, M, P)``: the volume integral of the convective flux, Eq. 1.
 * ``*_bruteforce``: the same operators through the explicit Kronecker matrix (or, for
-  ``convection``, the un-lifted sum of the paper's listing).
+  ``convection``, the three explicit Kronecker matrices of Eq. 1).
 * ``*_ld``: the same operators with every intermediate in ``long double``.
 """
 from __future__ import annotations
@@ -252,14 +252,15 @@ def convection(Dvq, Ivq, M, P, threads: int = 0) -> np.ndarray:
 
 
 def convection_bruteforce(Dvq, Ivq, M, P) -> np.ndarray:
-    """The same operator as one un-lifted sum over (l,m,n) per output (tiny sizes only)."""
+    """The same operator through the three explicit Kronecker matrices of Eq. 1, I⊗I⊗D, I⊗D⊗I
+    and D⊗I⊗I (tiny sizes only)."""
     Dvq, Ivq, M, P, nq, nv, E = _check_convection(Dvq, Ivq, M, P)
     if nq > 6 or nv > 6:
         raise ValueError("brute force is meant for tiny shapes")
     F = np.empty((3, E, nv, nv, nv), dtype=np.float64)
-    if E:
-        _load().oracle_convection_bruteforce_f64(_ptr(Dvq), _ptr(Ivq), _ptr(M), _ptr(P), _ptr(F),
-                                                 nq, nv, E)
+    if E and _load().oracle_convection_bruteforce_f64(_ptr(Dvq), _ptr(Ivq), _ptr(M), _ptr(P),
+                                                      _ptr(F), nq, nv, E):
+        raise MemoryError("oracle scratch allocation failed")
     return F
 
 

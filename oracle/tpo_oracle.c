@@ -263,35 +263,6 @@ int oracle_convection_f64(const double *Dvq, const double *Ivq, const double *M,
     return fail ? -1 : 0;
 }
 
-/* The same operator as the listing states it: one un-lifted sum over (l,m,n) per output. */
-int oracle_convection_bruteforce_f64(const double *Dvq, const double *Ivq, const double *M,
-                                     const double *P, double *F, int nq, int nv, long long E)
-{
-    const size_t q3 = (size_t)nq * nq * nq;
-    for (int c = 0; c < 3; ++c)
-        for (long long e = 0; e < E; ++e)
-            for (int k = 0; k < nv; ++k)
-                for (int j = 0; j < nv; ++j)
-                    for (int i = 0; i < nv; ++i) {
-                        double s = 0.0;
-                        for (int n = 0; n < nq; ++n)
-                            for (int m = 0; m < nq; ++m)
-                                for (int l = 0; l < nq; ++l) {
-                                    const size_t y = ((size_t)n * nq + m) * nq + l;
-                                    const double Me = M[(size_t)e * q3 + y];
-                                    const double *Pc = P + ((size_t)c * 3 * E + e) * q3 + y;
-                                    s = s + Dvq[i * nq + l] * Ivq[j * nq + m] * Ivq[k * nq + n] *
-                                                Me * Pc[0]
-                                          + Ivq[i * nq + l] * Dvq[j * nq + m] * Ivq[k * nq + n] *
-                                                Me * Pc[(size_t)E * q3]
-                                          + Ivq[i * nq + l] * Ivq[j * nq + m] * Dvq[k * nq + n] *
-                                                Me * Pc[2 * (size_t)E * q3];
-                                }
-                        F[(((size_t)c * E + e) * nv + k) * nv * nv + (size_t)j * nv + i] = s;
-                    }
-    return 0;
-}
-
 /* ---- the un-lifted definition ------------------------------------------- */
 
 /* K[(i m1 + j) m2 + k , (l n1 + m) n2 + n] = A[i,l] B[j,m] C[k,n]           */
@@ -320,6 +291,40 @@ static void matvec(const double *K, const double *x, double *y, size_t rows, siz
         for (size_t c = 0; c < cols; ++c) s = s + K[r * cols + c] * x[c];
         y[r] = s;
     }
+}
+
+/*
+ * The convective-flux integral without lifting, from the Kronecker form of Eq. 1: the three
+ * explicit matrices K0 = I (x) I (x) D, K1 = I (x) D (x) I, K2 = D (x) I (x) I (each nv^3 x nq^3)
+ * are built entry by entry and applied to vec(M[e] o P[c,d,e]); tiny sizes only.
+ */
+int oracle_convection_bruteforce_f64(const double *Dvq, const double *Ivq, const double *M,
+                                     const double *P, double *F, int nq, int nv, long long E)
+{
+    const size_t q3 = (size_t)nq * nq * nq, v3 = (size_t)nv * nv * nv;
+    double *K[3];
+    K[0] = kron3(Ivq, Ivq, Dvq, nq, nq, nq, nv, nv, nv);
+    K[1] = kron3(Ivq, Dvq, Ivq, nq, nq, nq, nv, nv, nv);
+    K[2] = kron3(Dvq, Ivq, Ivq, nq, nq, nq, nv, nv, nv);
+    double *x = (double *)malloc(q3 * sizeof(double) + 8);
+    double *t = (double *)malloc(v3 * sizeof(double) + 8);
+    int rc = -1;
+    if (K[0] && K[1] && K[2] && x && t) {
+        for (int c = 0; c < 3; ++c)
+            for (long long e = 0; e < E; ++e) {
+                double *Fe = F + ((size_t)c * E + e) * v3;
+                for (size_t y = 0; y < v3; ++y) Fe[y] = 0.0;
+                for (int d = 0; d < 3; ++d) {
+                    const double *Pd = P + (((size_t)c * 3 + d) * E + e) * q3;
+                    for (size_t y = 0; y < q3; ++y) x[y] = M[(size_t)e * q3 + y] * Pd[y];
+                    matvec(K[d], x, t, v3, q3);
+                    for (size_t y = 0; y < v3; ++y) Fe[y] = Fe[y] + t[y];
+                }
+            }
+        rc = 0;
+    }
+    free(K[0]); free(K[1]); free(K[2]); free(x); free(t);
+    return rc;
 }
 
 /* v[e] = kron(A,B,C) vec(u[e]) with the explicit matrix; tiny sizes only.   */

@@ -212,6 +212,16 @@ ekl_tpo_status ekl_tpo_apply_host(const double* A, const double* B, const double
                                   long long E, void* workspace, size_t workspace_bytes,
                                   cudaStream_t stream);
 
+/* Single-precision twins of the two host-buffer variants (same rules, float buffers). */
+ekl_tpo_status ekl_tpo_inv_helmholtz_host_f32(const float* S, const float* D, const float* u,
+                                              float* v, int n, long long E, void* workspace,
+                                              size_t workspace_bytes, cudaStream_t stream);
+ekl_tpo_status ekl_tpo_apply_host_f32(const float* A, const float* B, const float* C,
+                                      const float* u, float* v,
+                                      int n0, int n1, int n2, int m0, int m1, int m2,
+                                      long long E, void* workspace, size_t workspace_bytes,
+                                      cudaStream_t stream);
+
 /*
  * Bytes of device workspace that let the host-buffer variants run with chunks of
  * `chunk` elements: `n_inputs` per-element input fields of `in_elems_per_element`
@@ -282,6 +292,16 @@ int ekl_tpo_last_cuda_error(void);
  * SYNCHRONISES the device.  (Infrastructure: the paper has no counterpart.)
  */
 int ekl_tpo_device_error_flags(void);
+
+/*
+ * Self-test of that reporting path (infrastructure: the paper has no counterpart).  Enqueues
+ * one warp that waits on a barrier for a copy nobody issued.  Every wait in the library's
+ * kernels has a time budget of about one second; this one runs out of it twice (the wait and
+ * the bounded re-wait that follows a failure), so the kernel ends by itself after about two
+ * seconds and ekl_tpo_device_error_flags() then reports bit 0 once.  Nothing faults and the
+ * context stays usable.
+ */
+ekl_tpo_status ekl_tpo_selftest_expired_wait(cudaStream_t stream);
 
 /*
  * Measurement helper (no counterpart in the paper): enqueues `blocks` CTAs of 256

@@ -127,6 +127,65 @@ ekl_tpo_status pipeline(const T* const* mats, const size_t* mat_elems, int n_mat
     return EKL_TPO_OK;
 }
 
+template <typename T>
+ekl_tpo_status inv_helmholtz_host_impl(const T* S, const T* D, const T* u, T* v, int n,
+                                       long long E, void* workspace, size_t workspace_bytes,
+                                       cudaStream_t stream) {
+    if (n < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
+    if (E == 0) return EKL_TPO_OK;
+    if (!S || !D || !u || !v || !workspace) return EKL_TPO_ERR_NULL;
+    if (n > ekl::max_cubic_extent(sizeof(T))) return EKL_TPO_ERR_UNSUPPORTED;
+    const uintptr_t a = sizeof(T);
+    if (reinterpret_cast<uintptr_t>(S) % a || reinterpret_cast<uintptr_t>(D) % a ||
+        reinterpret_cast<uintptr_t>(u) % a || reinterpret_cast<uintptr_t>(v) % a)
+        return EKL_TPO_ERR_ALIGN;
+    const size_t n3 = (size_t)n * n * n;
+    const size_t field = (size_t)E * n3 * sizeof(T);
+    if (overlaps(v, field, S, (size_t)n * n * sizeof(T)) || overlaps(v, field, D, field) ||
+        (v != u && overlaps(v, field, u, field)))
+        return EKL_TPO_ERR_OVERLAP;
+    const T* mats[1] = {S};
+    const size_t mat_elems[1] = {(size_t)n * n};
+    const T* fin[2] = {D, u};
+    return pipeline<T>(
+        mats, mat_elems, 1, fin, 2, n3, v, n3, E, workspace, workspace_bytes, stream,
+        [n](T* const* dm, T* const* din, T* dout, long long cnt, cudaStream_t st) {
+            return ekl::launch_inv_helmholtz<T>(dm[0], din[0], din[1], dout, n, cnt, st);
+        });
+}
+
+template <typename T>
+ekl_tpo_status apply_host_impl(const T* A, const T* B, const T* C, const T* u, T* v, int n0,
+                               int n1, int n2, int m0, int m1, int m2, long long E,
+                               void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (n0 < 1 || n1 < 1 || n2 < 1 || m0 < 1 || m1 < 1 || m2 < 1 || E < 0)
+        return EKL_TPO_ERR_SHAPE;
+    if (E == 0) return EKL_TPO_OK;
+    if (!A || !B || !C || !u || !v || !workspace) return EKL_TPO_ERR_NULL;
+    if (!ekl::apply_fits(n0, n1, n2, m0, m1, m2, sizeof(T))) return EKL_TPO_ERR_UNSUPPORTED;
+    const uintptr_t a = sizeof(T);
+    if (reinterpret_cast<uintptr_t>(A) % a || reinterpret_cast<uintptr_t>(B) % a ||
+        reinterpret_cast<uintptr_t>(C) % a || reinterpret_cast<uintptr_t>(u) % a ||
+        reinterpret_cast<uintptr_t>(v) % a)
+        return EKL_TPO_ERR_ALIGN;
+    const size_t nout = (size_t)E * m0 * m1 * m2 * sizeof(T);
+    if (overlaps(v, nout, u, (size_t)E * n0 * n1 * n2 * sizeof(T)) ||
+        overlaps(v, nout, A, (size_t)m0 * n0 * sizeof(T)) ||
+        overlaps(v, nout, B, (size_t)m1 * n1 * sizeof(T)) ||
+        overlaps(v, nout, C, (size_t)m2 * n2 * sizeof(T)))
+        return EKL_TPO_ERR_OVERLAP;
+    const T* mats[3] = {A, B, C};
+    const size_t mat_elems[3] = {(size_t)m0 * n0, (size_t)m1 * n1, (size_t)m2 * n2};
+    const T* fin[2] = {u, nullptr};
+    return pipeline<T>(
+        mats, mat_elems, 3, fin, 1, (size_t)n0 * n1 * n2, v, (size_t)m0 * m1 * m2, E, workspace,
+        workspace_bytes, stream,
+        [=](T* const* dm, T* const* din, T* dout, long long cnt, cudaStream_t st) {
+            return ekl::launch_apply<T>(dm[0], dm[1], dm[2], din[0], dout, n0, n1, n2, m0, m1,
+                                             m2, cnt, st);
+        });
+}
+
 }  // namespace
 
 extern "C" {
@@ -147,59 +206,29 @@ size_t ekl_tpo_host_workspace_bytes(long long in_elems_per_element, int n_inputs
 ekl_tpo_status ekl_tpo_inv_helmholtz_host(const double* S, const double* D, const double* u,
                                           double* v, int n, long long E, void* workspace,
                                           size_t workspace_bytes, cudaStream_t stream) {
-    if (n < 1 || E < 0) return EKL_TPO_ERR_SHAPE;
-    if (E == 0) return EKL_TPO_OK;
-    if (!S || !D || !u || !v || !workspace) return EKL_TPO_ERR_NULL;
-    if (n > ekl::max_cubic_extent(sizeof(double))) return EKL_TPO_ERR_UNSUPPORTED;
-    const uintptr_t a = sizeof(double);
-    if (reinterpret_cast<uintptr_t>(S) % a || reinterpret_cast<uintptr_t>(D) % a ||
-        reinterpret_cast<uintptr_t>(u) % a || reinterpret_cast<uintptr_t>(v) % a)
-        return EKL_TPO_ERR_ALIGN;
-    const size_t n3 = (size_t)n * n * n;
-    const size_t field = (size_t)E * n3 * sizeof(double);
-    if (overlaps(v, field, S, (size_t)n * n * sizeof(double)) || overlaps(v, field, D, field) ||
-        (v != u && overlaps(v, field, u, field)))
-        return EKL_TPO_ERR_OVERLAP;
-    const double* mats[1] = {S};
-    const size_t mat_elems[1] = {(size_t)n * n};
-    const double* fin[2] = {D, u};
-    return pipeline<double>(
-        mats, mat_elems, 1, fin, 2, n3, v, n3, E, workspace, workspace_bytes, stream,
-        [n](double* const* dm, double* const* din, double* dout, long long cnt, cudaStream_t st) {
-            return ekl::launch_inv_helmholtz<double>(dm[0], din[0], din[1], dout, n, cnt, st);
-        });
+    return inv_helmholtz_host_impl<double>(S, D, u, v, n, E, workspace, workspace_bytes, stream);
+}
+
+ekl_tpo_status ekl_tpo_inv_helmholtz_host_f32(const float* S, const float* D, const float* u,
+                                              float* v, int n, long long E, void* workspace,
+                                              size_t workspace_bytes, cudaStream_t stream) {
+    return inv_helmholtz_host_impl<float>(S, D, u, v, n, E, workspace, workspace_bytes, stream);
 }
 
 ekl_tpo_status ekl_tpo_apply_host(const double* A, const double* B, const double* C,
                                   const double* u, double* v, int n0, int n1, int n2, int m0,
                                   int m1, int m2, long long E, void* workspace,
                                   size_t workspace_bytes, cudaStream_t stream) {
-    if (n0 < 1 || n1 < 1 || n2 < 1 || m0 < 1 || m1 < 1 || m2 < 1 || E < 0)
-        return EKL_TPO_ERR_SHAPE;
-    if (E == 0) return EKL_TPO_OK;
-    if (!A || !B || !C || !u || !v || !workspace) return EKL_TPO_ERR_NULL;
-    if (!ekl::apply_fits(n0, n1, n2, m0, m1, m2, sizeof(double))) return EKL_TPO_ERR_UNSUPPORTED;
-    const uintptr_t a = sizeof(double);
-    if (reinterpret_cast<uintptr_t>(A) % a || reinterpret_cast<uintptr_t>(B) % a ||
-        reinterpret_cast<uintptr_t>(C) % a || reinterpret_cast<uintptr_t>(u) % a ||
-        reinterpret_cast<uintptr_t>(v) % a)
-        return EKL_TPO_ERR_ALIGN;
-    const size_t nout = (size_t)E * m0 * m1 * m2 * sizeof(double);
-    if (overlaps(v, nout, u, (size_t)E * n0 * n1 * n2 * sizeof(double)) ||
-        overlaps(v, nout, A, (size_t)m0 * n0 * sizeof(double)) ||
-        overlaps(v, nout, B, (size_t)m1 * n1 * sizeof(double)) ||
-        overlaps(v, nout, C, (size_t)m2 * n2 * sizeof(double)))
-        return EKL_TPO_ERR_OVERLAP;
-    const double* mats[3] = {A, B, C};
-    const size_t mat_elems[3] = {(size_t)m0 * n0, (size_t)m1 * n1, (size_t)m2 * n2};
-    const double* fin[2] = {u, nullptr};
-    return pipeline<double>(
-        mats, mat_elems, 3, fin, 1, (size_t)n0 * n1 * n2, v, (size_t)m0 * m1 * m2, E, workspace,
-        workspace_bytes, stream,
-        [=](double* const* dm, double* const* din, double* dout, long long cnt, cudaStream_t st) {
-            return ekl::launch_apply<double>(dm[0], dm[1], dm[2], din[0], dout, n0, n1, n2, m0, m1,
-                                             m2, cnt, st);
-        });
+    return apply_host_impl<double>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, workspace,
+                                   workspace_bytes, stream);
+}
+
+ekl_tpo_status ekl_tpo_apply_host_f32(const float* A, const float* B, const float* C,
+                                      const float* u, float* v, int n0, int n1, int n2, int m0,
+                                      int m1, int m2, long long E, void* workspace,
+                                      size_t workspace_bytes, cudaStream_t stream) {
+    return apply_host_impl<float>(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, workspace,
+                                  workspace_bytes, stream);
 }
 
 }  // extern "C"

@@ -130,10 +130,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
                  : "memory");
 }
 
-// Bounded wait on a phase of the barrier; false if it gave up.
+// How long a wait on a bulk copy may last before it gives up (a copy takes microseconds).
+constexpr unsigned long long kWaitBudgetNs = 1000ull * 1000ull * 1000ull;
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait on a phase of the barrier; false if it gave up after about a second (the
+// clock is read every 256 polls).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
     const uint32_t a = smem_addr(bar);
-    for (unsigned it = 0; it < (1u << 24); ++it) {
+    unsigned long long t0 = 0;
+    for (unsigned it = 1;; ++it) {
         unsigned done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -143,8 +154,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
             : "r"(a), "r"(parity)
             : "memory");
         if (done) return true;
+        if ((it & 255u) == 0) {
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0)
+                t0 = now;
+            else if (now - t0 > kWaitBudgetNs)
+                return false;
+        }
     }
-    return false;
 }
 
 // Plain (non-multicast) bulk copy global -> this CTA's shared memory, completing on `bar`.

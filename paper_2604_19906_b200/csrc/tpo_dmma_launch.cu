@@ -1,4 +1,6 @@
 // Instances and launchers of the tensor-path kernels.
+#include "../../include/ekl_tpo.h"
+
 #include <cstdint>
 
 #include "dispatch.h"
@@ -300,6 +302,30 @@ template bool try_launch_apply_dmma<float>(const float*, const float*, const flo
                                            cudaStream_t, cudaError_t*);
 
 }  // namespace ekl
+
+namespace {
+// One warp arms a barrier for 16 bytes that nothing ever sends and waits for them: the wait
+// runs out of its time budget, raises bit 0 of the error flags and the kernel returns.
+__global__ void expired_wait_kernel() {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ekl::dmma::mbar_init(&bar, 1);
+        ekl::dmma::mbar_expect_tx(&bar, 16);
+    }
+    __syncthreads();
+    ekl::dmma::wait_bulk(&bar, 0);
+}
+}  // namespace
+
+extern "C" ekl_tpo_status ekl_tpo_selftest_expired_wait(cudaStream_t stream) {
+    expired_wait_kernel<<<1, 32, 0, stream>>>();
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) {
+        ekl::set_last_cuda_error((int)err);
+        return EKL_TPO_ERR_CUDA;
+    }
+    return EKL_TPO_OK;
+}
 
 // Reads (and clears) the flags device code raises when something that should never happen
 // did: bit 0 = a bounded wait on a bulk copy gave up, bit 1 = a launch's ticket counter was

@@ -231,28 +231,39 @@ def _declare_host(lib):
     lib.ekl_tpo_inv_helmholtz_host.restype = i
     lib.ekl_tpo_apply_host.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, i, i, ll, vp, sz, vp]
     lib.ekl_tpo_apply_host.restype = i
+    lib.ekl_tpo_inv_helmholtz_host_f32.argtypes = lib.ekl_tpo_inv_helmholtz_host.argtypes
+    lib.ekl_tpo_inv_helmholtz_host_f32.restype = i
+    lib.ekl_tpo_apply_host_f32.argtypes = lib.ekl_tpo_apply_host.argtypes
+    lib.ekl_tpo_apply_host_f32.restype = i
     lib.ekl_tpo_host_workspace_bytes.argtypes = [ll, i, ll, ll, ll, i]
     lib.ekl_tpo_host_workspace_bytes.restype = sz
     lib._host_declared = True
 
 
 def host_workspace(device, nbytes: int) -> torch.Tensor:
-    """A cached device scratch buffer of at least ``nbytes`` bytes on ``device`` (device
-    memory comes from torch; the library itself allocates none)."""
+    """A cached device scratch buffer of at least ``nbytes`` bytes for host-buffer calls on the
+    current stream of ``device`` (device memory comes from torch; the library itself allocates
+    none).  One buffer per (device, stream): calls that share a workspace must be ordered on
+    one stream.  The library also works on the buffer from two helper streams that torch's
+    allocator does not know of, so before a buffer is replaced by a larger one the stream it
+    served is synchronised -- the last call's copies have then left it."""
     dev = torch.device(device)
-    key = (dev.type, dev.index)
+    stream = torch.cuda.current_stream(dev)
+    key = (dev.type, dev.index, stream.cuda_stream)
     ws = _workspaces.get(key)
     if ws is None or ws.numel() < nbytes:
+        if ws is not None:
+            stream.synchronize()
         ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
         _workspaces[key] = ws
     return ws
 
 
-def _host_ptr(t: torch.Tensor, name: str) -> int:
+def _host_ptr(t: torch.Tensor, name: str, dtype: torch.dtype = torch.float64) -> int:
     if not isinstance(t, torch.Tensor) or t.is_cuda:
         raise TypeError(f"{name} must be a CPU tensor")
-    if t.dtype != torch.float64:
-        raise TypeError(f"{name} must be float64")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}")
     if not t.is_contiguous():
         raise ValueError(f"{name} must be contiguous (row-major)")
     return t.data_ptr()
@@ -261,22 +272,27 @@ def _host_ptr(t: torch.Tensor, name: str) -> int:
 def ekl_tpo_inv_helmholtz_host(S, D, u, out, device="cuda:0", chunk: int = 2048,
                                workspace: torch.Tensor | None = None):
     """Inverse Helmholtz with HOST tensors in and out (pinned memory lets copies and
-    kernels overlap).  Enqueues on the current stream of ``device`` and returns; the
-    result is complete once that stream has been synchronised."""
+    kernels overlap), float64 or float32 (the dtype of ``u`` decides).  Enqueues on the current
+    stream of ``device`` and returns; the result is complete once that stream has been
+    synchronised."""
     lib = library()
     _declare_host(lib)
+    dtype = u.dtype
+    if dtype not in (torch.float64, torch.float32):
+        raise TypeError("u must be float64 or float32")
+    w = 8 if dtype == torch.float64 else 4
+    fn = lib.ekl_tpo_inv_helmholtz_host if w == 8 else lib.ekl_tpo_inv_helmholtz_host_f32
     E, n = u.shape[0], S.shape[0]
     if tuple(S.shape) != (n, n) or tuple(u.shape[1:]) != (n, n, n) or D.shape != u.shape \
             or out.shape != u.shape:
         raise ValueError("expected S [n,n] and D,u,out [E,n,n,n]")
     dev = torch.device(device)
     if workspace is None:
-        need = lib.ekl_tpo_host_workspace_bytes(n ** 3, 2, n ** 3, n * n, max(1, min(chunk, E)), 8)
+        need = lib.ekl_tpo_host_workspace_bytes(n ** 3, 2, n ** 3, n * n, max(1, min(chunk, E)), w)
         workspace = host_workspace(dev, need)
-    ptrs = [_host_ptr(t, nm) for t, nm in ((S, "S"), (D, "D"), (u, "u"), (out, "out"))]
+    ptrs = [_host_ptr(t, nm, dtype) for t, nm in ((S, "S"), (D, "D"), (u, "u"), (out, "out"))]
     with torch.cuda.device(dev):
-        st = lib.ekl_tpo_inv_helmholtz_host(*ptrs, n, E, workspace.data_ptr(), workspace.numel(),
-                                            _stream(dev))
+        st = fn(*ptrs, n, E, workspace.data_ptr(), workspace.numel(), _stream(dev))
     if st:
         raise EklTpoError(st, "ekl_tpo_inv_helmholtz_host")
     return out
@@ -288,6 +304,11 @@ def ekl_tpo_apply_host(A, B, C, u, out, device="cuda:0", chunk: int = 4096,
     :func:`ekl_tpo_inv_helmholtz_host`."""
     lib = library()
     _declare_host(lib)
+    dtype = u.dtype
+    if dtype not in (torch.float64, torch.float32):
+        raise TypeError("u must be float64 or float32")
+    w = 8 if dtype == torch.float64 else 4
+    fn = lib.ekl_tpo_apply_host if w == 8 else lib.ekl_tpo_apply_host_f32
     (m0, n0), (m1, n1), (m2, n2) = A.shape, B.shape, C.shape
     E = u.shape[0]
     if tuple(u.shape[1:]) != (n0, n1, n2) or tuple(out.shape) != (E, m0, m1, m2):
@@ -296,12 +317,13 @@ def ekl_tpo_apply_host(A, B, C, u, out, device="cuda:0", chunk: int = 4096,
     if workspace is None:
         need = lib.ekl_tpo_host_workspace_bytes(n0 * n1 * n2, 1, m0 * m1 * m2,
                                                 m0 * n0 + m1 * n1 + m2 * n2,
-                                                max(1, min(chunk, E)), 8)
+                                                max(1, min(chunk, E)), w)
         workspace = host_workspace(dev, need)
-    ptrs = [_host_ptr(t, nm) for t, nm in ((A, "A"), (B, "B"), (C, "C"), (u, "u"), (out, "out"))]
+    ptrs = [_host_ptr(t, nm, dtype)
+            for t, nm in ((A, "A"), (B, "B"), (C, "C"), (u, "u"), (out, "out"))]
     with torch.cuda.device(dev):
-        st = lib.ekl_tpo_apply_host(*ptrs, n0, n1, n2, m0, m1, m2, E, workspace.data_ptr(),
-                                    workspace.numel(), _stream(dev))
+        st = fn(*ptrs, n0, n1, n2, m0, m1, m2, E, workspace.data_ptr(), workspace.numel(),
+                _stream(dev))
     if st:
         raise EklTpoError(st, "ekl_tpo_apply_host")
     return out

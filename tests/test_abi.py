@@ -155,3 +155,22 @@ def test_product_never_imports_the_oracle():
     for path in glob.glob(os.path.join(ROOT, "oracle", "*")):
         if path.endswith((".py", ".c", ".h")):
             assert "paper_2604_19906_b200" not in open(path).read(), path
+
+
+def test_header_compiles_as_c_and_validation_answers_from_a_c_program(lib, tmp_path):
+    """gcc (a C compiler, not nvcc) sees include/ekl_tpo.h and links the library."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    cuda_inc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "include")
+    if not gcc or not os.path.exists(os.path.join(cuda_inc, "cuda_runtime_api.h")):
+        pytest.skip("gcc or the CUDA headers are not available")
+    libdir = os.path.join(ROOT, "paper_2604_19906_b200", "lib")
+    exe = str(tmp_path / "abi_check")
+    subprocess.run([gcc, "-std=c11", "-Wall", "-Wextra", "-Werror",
+                    "-I", os.path.join(ROOT, "include"), "-I", cuda_inc,
+                    os.path.join(ROOT, "tests", "c_abi", "abi_check.c"), "-o", exe,
+                    "-L", libdir, "-lekl_tpo", f"-Wl,-rpath,{libdir}"], check=True)
+    r = subprocess.run([exe], capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "abi_check: ok" in r.stdout

@@ -62,6 +62,31 @@ def test_apply_host_matches_oracle(env):
     assert oracle.rel_err_per_element(out.numpy(), want).max() <= 1e-12
 
 
+@pytest.mark.parametrize("n,E,chunk", [(14, 203, 40), (7, 100, 13), (22, 5, 2)])
+def test_host_variants_in_single_precision(env, n, E, chunk):
+    torch, ops, oracle = env["torch"], env["ops"], env["oracle"]
+    g = np.random.Generator(np.random.PCG64(900 + n))
+    S = np.linalg.qr(g.standard_normal((n, n)))[0].astype(np.float32)
+    D = g.uniform(0.1, 1.3, (E, n, n, n)).astype(np.float32)
+    u = g.uniform(-1, 1, (E, n, n, n)).astype(np.float32)
+    want = oracle.inv_helmholtz(S, D, u)                  # the oracle widens and works in fp64
+    h = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in (S, D, u)]
+    out = torch.full((E, n, n, n), float("nan"), dtype=torch.float32).pin_memory()
+    ops.ekl_tpo_inv_helmholtz_host(*h, out, device=env["dev"], chunk=chunk)
+    torch.cuda.synchronize()
+    assert oracle.rel_err_per_element(out.numpy(), want).max() <= 1e-5
+    nn, mm = (8, 8, 8), (12, 12, 12)
+    A, B, C = (g.standard_normal((mm[d], nn[d])).astype(np.float32) / np.float32(np.sqrt(8.0))
+               for d in range(3))
+    ua = g.uniform(-1, 1, (E,) + nn).astype(np.float32)
+    wanta = oracle.tpo_apply(A, B, C, ua)
+    ha = [torch.from_numpy(np.ascontiguousarray(x)).pin_memory() for x in (A, B, C, ua)]
+    outa = torch.full((E,) + mm, float("nan"), dtype=torch.float32).pin_memory()
+    ops.ekl_tpo_apply_host(*ha, outa, device=env["dev"], chunk=chunk)
+    torch.cuda.synchronize()
+    assert oracle.rel_err_per_element(outa.numpy(), wanta).max() <= 1e-5
+
+
 def test_host_workspace_rules(env):
     torch, ops = env["torch"], env["ops"]
     lib = ops.library()

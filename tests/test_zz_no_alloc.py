@@ -94,3 +94,32 @@ def test_static_variant_rejects_batches_beyond_its_maximum(env):
     with torch.cuda.device(dev):
         assert fn(None, None, None, None, n, 0, None) == 0
         assert fn(S.data_ptr(), D.data_ptr(), u.data_ptr(), got.data_ptr(), 0, 5, None) == 2
+
+
+def test_static_variant_against_the_oracle_odd_and_large_extents_in_place_and_queued(env):
+    """Directly against the CPU oracle (not only against the workspace variant): an odd extent,
+    an extent that takes the general kernel, v == u on pinned memory, and two calls of
+    different sizes queued on one stream with a single synchronise, which is the documented
+    way to share the staging area."""
+    import oracle
+    torch, ops, dev = env["torch"], env["ops"], env["dev"]
+    cases = []
+    for n, E, seed in ((5, 41, 11), (22, 9, 12), (14, 65, 13), (3, 7, 14)):
+        S, D, u = make_case(torch, n, E, seed)
+        want = oracle.inv_helmholtz(S.numpy(), D.numpy(), u.numpy())
+        cases.append((S, D, u, want))
+    # queued back to back, one synchronise at the end
+    outs = [torch.full(c[2].shape, float("nan"), dtype=torch.float64).pin_memory() for c in cases]
+    for (S, D, u, _), out in zip(cases, outs):
+        ops.ekl_tpo_inv_helmholtz_host_static(S, D, u, out, device=dev)
+    torch.cuda.synchronize()
+    for (S, D, u, want), out in zip(cases, outs):
+        assert oracle.rel_err_per_element(out.numpy(), want).max() <= TOL64
+    # in place: v == u
+    S, D, u, want = cases[0]
+    inplace = u.clone().pin_memory()
+    ops.ekl_tpo_inv_helmholtz_host_static(S, D, inplace, inplace, device=dev)
+    torch.cuda.synchronize()
+    assert np.array_equal(inplace.numpy(), outs[0].numpy())
+    # the status code cannot see a device-side wait that gave up; the flags can
+    assert ops.library().ekl_tpo_device_error_flags() == 0

@@ -303,17 +303,6 @@ int ekl_tpo_device_error_flags(void);
  */
 ekl_tpo_status ekl_tpo_selftest_expired_wait(cudaStream_t stream);
 
-/*
- * Measurement helper (no counterpart in the paper): enqueues `blocks` CTAs of 256
- * threads, each thread running 16 independent chains of `iters` dependent fp64 FMAs
- * in registers, and stores in *flops (HOST pointer, written before returning) the
- * number of floating-point operations that launch performs.  `sink` is a device
- * buffer of at least blocks*256 doubles that receives one value per thread.  Timing
- * the launch gives the sustained FP64 FMA rate the roofline fractions refer to.
- */
-ekl_tpo_status ekl_tpo_probe_fp64_fma(double* sink, int blocks, int iters, double* flops,
-                                      cudaStream_t stream);
-
 #ifdef __cplusplus
 }
 #endif

@@ -2,6 +2,7 @@
 
 ``lib/libekl_tpo.so``    the product: C-ABI operators (``include/ekl_tpo.h``)
 ``lib/libekl_inputs.so`` device twin of the seeded input stream (``inputs.py``)
+``lib/libekl_probe.so``  measurement helpers (``include/ekl_probe.h``), not on the product path
 
 Objects go to ``_build/`` (not tracked).  Only sources newer than their object are
 recompiled; any header change recompiles everything.
@@ -26,6 +27,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 LIBS = {
     "libekl_inputs.so": ["inputs_fill.cu"],
+    "libekl_probe.so": ["peak_probe.cu"],
     # every other .cu under csrc/ belongs to the product library
 }
 

@@ -89,7 +89,7 @@ template <int NQ, int NV>
 __global__ void __launch_bounds__(ConvCfg<NQ, NV>::kThreads, ConvCfg<NQ, NV>::kCtasPerSm)
 convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
                 const double* __restrict__ M, const double* __restrict__ P, double* __restrict__ F,
-                long long E) {
+                long long E, unsigned long long* tickets) {
     using C = ConvCfg<NQ, NV>;
     using S1 = typename C::S1;
     using S2 = typename C::S2;
@@ -109,6 +109,10 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
     load_op<S1, double>(opI, Ivq, true, lane);
     load_op<S1, double>(opD, Dvq, true, lane);
 
+    // elements are handed out one at a time (BatchQueue, a batch being one element)
+    __shared__ long long shared_next;
+    BatchQueue q;
+    q.start(tickets, &shared_next);
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
 
@@ -128,24 +132,36 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
         }
     };
 
-    long long e = blockIdx.x;
-    if (threadIdx.x == 0 && e < E) fetch(0, e, true);
+    if (threadIdx.x == 0 && q.batch < E) fetch(0, q.batch, true);
     unsigned parity = 0;
-    for (; e < E; e += gridDim.x) {
-        // ask L2 for everything this element still needs and for the first fields of the
-        // next one, a whole element of work ahead of the bulk copies that will use them
+    bool ok = true;
+    while (ok && q.batch < E) {
+        q.draw();
+        const long long e = q.batch;
+        // ask L2 for everything this element still needs, a whole element of work ahead of
+        // the bulk copies that will use it
         if (threadIdx.x == 0) {
             const unsigned field = (unsigned)(kQ3 * sizeof(double));
             for (int cd = 3; cd < 9; ++cd) bulk_prefetch_l2(P + ((size_t)cd * E + e) * kQ3, field);
-            const long long ne = e + gridDim.x;
-            if (ne < E) {
-                bulk_prefetch_l2(M + (size_t)ne * kQ3, field);
-                for (int d = 0; d < 3; ++d) bulk_prefetch_l2(P + ((size_t)d * E + ne) * kQ3, field);
-            }
         }
         for (int c = 0; c < 3; ++c) {
-            if (!wait_bulk(bar, parity)) return;
+            if (!wait_bulk(bar, parity)) {
+                ok = false;
+                break;
+            }
             parity ^= 1u;
+            if (c == 0) {
+                // the barrier inside the wait orders the ticket handed over at the end of the
+                // previous element; now the next element is known: ask L2 for its first fields
+                q.refresh();
+                const long long ne = q.next;
+                if (threadIdx.x == 0 && ne < E) {
+                    const unsigned field = (unsigned)(kQ3 * sizeof(double));
+                    bulk_prefetch_l2(M + (size_t)ne * kQ3, field);
+                    for (int d = 0; d < 3; ++d)
+                        bulk_prefetch_l2(P + ((size_t)d * E + ne) * kQ3, field);
+                }
+            }
             // stage 1: three products, 3 * kTiles tile tasks dealt round-robin
 #pragma unroll
             for (int it = 0; it < (3 * S1::kTiles + C::kWarps - 1) / C::kWarps; ++it) {
@@ -162,7 +178,7 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             // the P buffers (and, after the last component, M) are free: fetch what comes next
             if (threadIdx.x == 0) {
                 const bool last = (c == 2);
-                const long long ne = last ? e + gridDim.x : e;
+                const long long ne = last ? q.next : e;
                 if (ne < E) {
                     fence_async_proxy();
                     fetch(last ? 0 : c + 1, ne, last);
@@ -203,7 +219,10 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             // the next stage 1 writes sT, which stage 2 no longer reads; the next stage 2
             // writes sW only after the barrier that follows the next stage 1
         }
+        q.publish();
+        q.advance_batch();
     }
+    q.finish(E);
 }
 
 }  // namespace dmma

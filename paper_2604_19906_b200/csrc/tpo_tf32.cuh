@@ -213,7 +213,9 @@ struct IhCfg32 {
     static constexpr int kByWarps = kMaxWarpsPerSm / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
-    static constexpr int kFactorDepth = (Mid::kTilesPerWarp >= 6) ? 4 : 2;
+    // tiles of the pointwise factor held ahead in registers: deeper than this spills at the
+    // 80 registers three CTAs per SM leave a thread (measured: n = 14 9 % and n = 8 12 % faster)
+    static constexpr int kFactorDepth = (N == 8) ? 1 : 2;
 };
 
 // v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])), fp32 fields; u must be 16-byte aligned.

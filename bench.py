@@ -44,10 +44,28 @@ SM_MAX_GHZ = 1.965
 FP64_PEAK_TFLOPS = SM_COUNT * FP64_LANES_PER_SM * 2 * SM_MAX_GHZ / 1e3
 HBM_FALLBACK_GBS = 6650.0
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per element of the operator
-# kernel, from the ncu captures summarised under profiles/ (taken on a smaller E of the same
-# kernel; traffic is proportional to the number of elements).  Workload index -> bytes.
-NCU_TRAFFIC_BYTES_PER_ELEMENT = {3: 67676.0, 4: 16200.0, 5: 150400.0, 6: 32590.0}
+# Nominal figures quoted for context beside the measured ones: HBM3e bandwidth and the FP64
+# rate of the data sheet.
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_FP64_TFLOPS = 40.0
+L2_BYTES = 126e6
+
+
+def ncu_traffic_bytes_per_element(wl_index: int):
+    """DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per element of the operator
+    kernel from the ncu capture recorded in profiles/dram_traffic.json (taken on a smaller E of
+    the same kernel; traffic is proportional to the number of elements).  None if there is no
+    capture for this workload or the kernel sources have changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            entry = json.load(f).get(f"cfg{wl_index}")
+        from paper_2604_19906_b200 import profile_summary
+        if entry and entry.get("source_digest") == profile_summary.source_digest():
+            return float(entry["bytes_per_element"])
+    except Exception:
+        pass
+    return None
 
 
 def measured_peaks():
@@ -135,21 +153,49 @@ def oracle_run(wl, e0, e1):
     return time.perf_counter() - t0, v, host
 
 
-def cpu_baseline(wl, target_seconds=12.0, max_elements=None):
-    """The oracle, as it stands, on all host cores over a bounded sample (the first Ns
-    elements) of the workload.  Returns the cpu_baseline object, the sample's output."""
+def oracle_call(wl, host, threads=0):
     import oracle
+    if wl.op == "inv_helmholtz":
+        return oracle.inv_helmholtz(host["S"], host["D"], host["u"], threads)
+    if wl.op == "convection":
+        return oracle.convection(host["Dvq"], host["Ivq"], host["M"], host["P"], threads)
+    return oracle.tpo_apply(host["A"], host["B"], host["C"], host["u"], threads)
+
+
+def cpu_baseline(wl, target_seconds=4.0, max_elements=None):
+    """The oracle, as it stands, on all host cores over a bounded sample (the first Ns
+    elements) of the workload: one untimed pass, then the best of three timed ones.  Also a
+    1-thread figure on (at most) the first 8192 elements -- the batch size and the "seq."
+    column of the paper's Table 2.  Returns the cpu_baseline object, the sample's output."""
+    import oracle
+    from paper_2604_19906_b200 import inputs
     probe = min(wl.E, 256)
     t_probe, _, _ = oracle_run(wl, 0, probe)
     rate = probe / max(t_probe, 1e-6)
     ns = int(min(wl.E, max(probe, rate * target_seconds)))
     if max_elements:
         ns = min(ns, max_elements)
-    t, v, _ = oracle_run(wl, 0, ns)
+    _, v, host = oracle_run(wl, 0, ns)                        # warm-up pass, keeps the output
+    times = []
+    for _ in range(3):
+        t0 = time.perf_counter()
+        oracle_call(wl, host)
+        times.append(time.perf_counter() - t0)
+    t = min(times)
     cores = oracle.threads_used(0)
+    n1 = min(wl.E, 8192, ns)
+    host1 = host if n1 == ns else inputs.host_case(wl, 0, n1)
+    oracle_call(wl, host1, 1)
+    t0 = time.perf_counter()
+    oracle_call(wl, host1, 1)
+    t1 = time.perf_counter() - t0
     return {"value": ns / t, "unit": UNIT, "cores": cores, "kind": "oracle",
             "gflops": ns * wl.flops_per_element / t / 1e9,
-            "sample": f"first {ns} of {wl.E} elements of {wl.name}, {t:.2f} s on {cores} threads"
+            "sample": f"first {ns} of {wl.E} elements of {wl.name}, best of 3 warm passes "
+                      f"({t:.2f} s) on {cores} threads",
+            "one_thread": {"value": n1 / t1, "unit": UNIT, "elements": n1,
+                           "ms": t1 * 1e3,
+                           "note": "1 thread; the paper's Table 2 times 8192-element batches"}
             }, v, ns
 
 
@@ -209,6 +255,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-probes", action="store_true",
+                    help="skip the FP64-rate probes that run after the timed region")
+    ap.add_argument("--context", action="store_true",
+                    help="add the E = 8192 rows (the batch size of the paper's Table 2) for "
+                         "n = 4, 8, 12, 14 to the line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -228,8 +279,9 @@ def main():
     # The oracle leg runs first, before any CUDA call (its OpenMP pool and the CUDA
     # context do not interact, and the GPUs are not held while the host works).
     base = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        base, v_oracle, ns_oracle = cpu_baseline(wl)
+    if rank == 0 and not args.no_cpu_baseline:
+        # under torchrun the other ranks wait at the first barrier: keep the sample small there
+        base, v_oracle, ns_oracle = cpu_baseline(wl, max_elements=None if world == 1 else 8192)
 
     import torch
     from paper_2604_19906_b200 import build, ops, sharding
@@ -324,31 +376,34 @@ def main():
                else v[:ns_oracle]).cpu().numpy().astype(np.float64)
         max_rel_err = float(oracle.rel_err_per_element(got, v_oracle).max())
 
-    # ---------------------------------------------------------------- FP64 rate of this device, live
-    fp64_meas = None
-    if rank == 0:
-        import ctypes
-        sink = torch.empty(SM_COUNT * 8 * 256, dtype=torch.float64, device=dev)
-        flops = ctypes.c_double(0.0)
-        with torch.cuda.stream(stream):
-            best = None
-            for it in range(4):
-                s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                s.record(stream)
-                lib.ekl_tpo_probe_fp64_fma.argtypes = None
-                rc = lib.ekl_tpo_probe_fp64_fma(ctypes.c_void_p(sink.data_ptr()), SM_COUNT * 8,
-                                                20000, ctypes.byref(flops), ctypes.c_void_p(sp))
-                e.record(stream)
-                torch.cuda.synchronize(dev)
-                if rc == 0 and it > 0:
-                    ms = s.elapsed_time(e)
-                    best = ms if best is None else min(best, ms)
-        if best:
-            fp64_meas = flops.value / (best * 1e-3) / 1e12
+    # ---------------------------------------------------------------- FP64 rates of this device, live
+    probe_rates = {}
+    if rank == 0 and not args.no_probes:
+        from paper_2604_19906_b200 import probes
+        try:
+            probe_rates = probes.run_probes(dev, stream)
+        except Exception as exc:                      # a missing probe library is not fatal here
+            probe_rates = {"error": str(exc)}
+
+    # ---------------------------------------------------------------- small workloads: cold and graph
+    small = None
+    if rank == 0 and E * wl.bytes_per_element < 2 * L2_BYTES:
+        small = small_workload_variants(torch, inputs, wl, fn, dev, stream, ops)
+        if small is not None and world == 1:
+            # the timed region above re-used one buffer set (warm L2); the headline of a
+            # workload that fits in L2 is the cold figure, each call on another buffer set
+            ms_per_step = small["cold_us"] / 1e3
+            value = E / (ms_per_step * 1e-3)
+            launch_ms = [ms_per_step]
+
+    # ---------------------------------------------------------------- E = 8192 context rows
+    context = None
+    if rank == 0 and args.context:
+        context = context_rows(torch, inputs, ops, dev, stream)
 
     # ---------------------------------------------------------------- end to end with host buffers
     e2e = None
-    if not args.no_e2e and wl.op != "convection" and wl.dtype == "f64":
+    if not args.no_e2e and wl.op != "convection":
         e2e = run_e2e(torch, ops, wl, case, dev, stream, args.e2e_steps, world, dist)
 
     if rank != 0:
@@ -357,6 +412,7 @@ def main():
         return
 
     peaks, peak_src = measured_peaks()
+    traffic_pe = ncu_traffic_bytes_per_element(wl.index)
     avg_launch_ms = statistics.fmean(launch_ms)
     flops_launch = E * wl.flops_per_element
     bytes_launch = E * wl.bytes_per_element
@@ -380,9 +436,10 @@ def main():
         roof = {"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s",
                 "frac": gbs / hbm_peak}
     roof.update({
-        "traffic": (NCU_TRAFFIC_BYTES_PER_ELEMENT[wl.index] * E
-                    if wl.index in NCU_TRAFFIC_BYTES_PER_ELEMENT else None),
-        "traffic_note": "bytes per launch: ncu dram read+write per element (profiles/) x E",
+        "traffic": (traffic_pe * E if traffic_pe is not None else None),
+        "traffic_note": "bytes per launch: ncu dram read+write per element "
+                        "(profiles/dram_traffic.json) x E; null if there is no capture of the "
+                        "current kernel sources",
         "algorithmic_bytes": bytes_launch, "algorithmic_flops": flops_launch,
         "kernel_ms": avg_launch_ms,
         "peak_source": ("alu: 148 SMs x 64 FP64 FMA/clk x 2 x 1.965 GHz; hbm: "
@@ -390,7 +447,19 @@ def main():
                         f"hbm: MEASURED_PEAKS.json ({peak_src}); tensor: bf16 x 1.1/2.25, "
                         "three TF32 steps per product"),
         "fp64_tflops": tf, "fp64_peak_derived": FP64_PEAK_TFLOPS,
-        "fp64_peak_probe_tflops": fp64_meas,
+        "fp64_peak_probe_tflops": probe_rates.get("fma_chain"),
+        "fp64_peak_probe_dfma_tflops": probe_rates.get("fma_contraction"),
+        "fp64_peak_probe_dmma_tflops": probe_rates.get("dmma_2chains"),
+        "fp64_peak_probe_dmma_plus_fma_tflops": probe_rates.get("dmma_plus_fma"),
+        "stage_loop_n14_dmma_tflops": probe_rates.get("stage_loop_n14_dmma"),
+        "stage_loop_n14_dmma_padded_tflops": probe_rates.get("stage_loop_n14_dmma_padded"),
+        "stage_loop_n14_fma_tflops": probe_rates.get("stage_loop_n14_fma"),
+        "nominal": {"hbm_gbs": NOMINAL_HBM_GBS, "fp64_tflops": NOMINAL_FP64_TFLOPS,
+                    "min_roof_ms": max(flops_launch / (NOMINAL_FP64_TFLOPS * 1e12),
+                                       bytes_launch / (NOMINAL_HBM_GBS * 1e9)) * 1e3,
+                    "frac_of_min_roof": max(flops_launch / (NOMINAL_FP64_TFLOPS * 1e12),
+                                            bytes_launch / (NOMINAL_HBM_GBS * 1e9)) * 1e3
+                    / avg_launch_ms} if wl.dtype == "f64" else None,
         "hbm_gbs": gbs, "hbm_peak_gbs": hbm_peak, "hbm_frac": gbs / hbm_peak,
         "min_roof_ms": max(t_alu, t_hbm) * 1e3,
         "frac_of_min_roof": max(t_alu, t_hbm) * 1e3 / avg_launch_ms})
@@ -399,7 +468,9 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "elements_per_gpu": E,
                        "l2": f"inputs larger than L2 ({bytes_launch / 1e9:.2f} GB per step)"
-                       if bytes_launch > 2 * 126e6 else "working set fits in L2 (warm)",
+                       if bytes_launch > 2 * L2_BYTES else
+                       (f"rotating over {small['sets']} buffer sets (3 x L2) between calls"
+                        if small is not None and world == 1 else "working set fits in L2 (warm)"),
                        "parallelism": f"elements sharded over {world} GPU(s), no collective"},
             "gflops": value * wl.flops_per_element / 1e9,
             "roofline": roof, "clocks": clocks, "gpu_launches": args.steps,
@@ -408,9 +479,108 @@ def main():
         line["cpu_baseline"] = base
     if e2e is not None:
         line["e2e"] = e2e
+    if small is not None:
+        line["small_workload"] = small
+    if context is not None:
+        line["paper_batch_8192"] = context
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def _event_ms(torch, stream, fn_once, reps):
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record(stream)
+    for k in range(reps):
+        fn_once(k)
+    s1.record(stream)
+    stream.synchronize()
+    return s0.elapsed_time(s1) / reps
+
+
+def small_workload_variants(torch, inputs, wl, fn, dev, stream, ops, reps=200):
+    """For a workload whose working set fits in L2 (configurations 0 and 1): microseconds per
+    call (a) warm, the same buffers every call, (b) cold, rotating over enough distinct buffer
+    sets to exceed three times the L2, (c) warm, replayed from a CUDA graph of 20 calls.  At
+    this size the call is at the scale of the launch path, not of either roof."""
+    if wl.op != "inv_helmholtz" or wl.dtype != "f64":
+        return None
+    n, E = wl.n[0], wl.E
+    base = inputs.device_case(wl, dev)
+    set_bytes = E * wl.bytes_per_element
+    sets = int(min(4096, max(3, -(-int(3 * L2_BYTES) // set_bytes))))
+    us = [base["u"]] + [base["u"].clone() for _ in range(sets - 1)]
+    Ds = [base["D"]] + [base["D"].clone() for _ in range(sets - 1)]
+    vs = [torch.empty_like(base["u"]) for _ in range(sets)]
+    sp = stream.cuda_stream
+
+    def call(k):
+        st = fn(base["S"].data_ptr(), Ds[k].data_ptr(), us[k].data_ptr(), vs[k].data_ptr(), n, E, sp)
+        if st:
+            raise ops.EklTpoError(st, "small workload step")
+
+    out = {"sets": sets, "bytes_per_set": set_bytes, "calls": reps}
+    with torch.cuda.stream(stream):
+        for k in range(sets):
+            call(k)
+        stream.synchronize()
+        out["warm_us"] = 1e3 * _event_ms(torch, stream, lambda k: call(0), reps)
+        out["cold_us"] = 1e3 * _event_ms(torch, stream, lambda k: call(k % sets), reps)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(20):
+                call(0)
+        graph.replay()
+        stream.synchronize()
+        out["graph_us"] = 1e3 * _event_ms(torch, stream, lambda k: graph.replay(), 10) / 20
+    flops, nbytes = E * wl.flops_per_element, set_bytes
+    peaks, _ = measured_peaks()
+    roof_us = 1e6 * max(flops / (FP64_PEAK_TFLOPS * 1e12),
+                        nbytes / (float(peaks.get("hbm_gbs", HBM_FALLBACK_GBS)) * 1e9))
+    out["roofline_us"] = roof_us
+    out["cold_frac_of_roof"] = roof_us / out["cold_us"]
+    out["note"] = "latency-limited: the roofline time is below the cost of one kernel launch"
+    return out
+
+
+def context_rows(torch, inputs, ops, dev, stream, reps=50):
+    """E = 8192 (the batch the paper's Table 2 measures on) at n = 4, 8, 12, 14, fp64 inverse
+    Helmholtz: milliseconds per call (rotating over buffer sets larger than L2) and the
+    oracle on one host thread beside it."""
+    import oracle
+    rows = []
+    lib = ops.library()
+    for n in (4, 8, 12, 14):
+        wl = inputs.Workload(1, "inv_helmholtz", (n, n, n), (n, n, n), 8192, "f64")
+        base = inputs.device_case(wl, dev)
+        set_bytes = wl.E * wl.bytes_per_element
+        sets = int(max(2, -(-int(3 * L2_BYTES) // set_bytes)))
+        us = [base["u"]] + [base["u"].clone() for _ in range(sets - 1)]
+        Ds = [base["D"]] + [base["D"].clone() for _ in range(sets - 1)]
+        v = torch.empty_like(base["u"])
+        sp = stream.cuda_stream
+
+        def call(k):
+            st = lib.ekl_tpo_inv_helmholtz(base["S"].data_ptr(), Ds[k % sets].data_ptr(),
+                                           us[k % sets].data_ptr(), v.data_ptr(), n, wl.E, sp)
+            if st:
+                raise ops.EklTpoError(st, "context row")
+
+        with torch.cuda.stream(stream):
+            for k in range(sets):
+                call(k)
+            stream.synchronize()
+            ms = _event_ms(torch, stream, call, reps)
+        host = inputs.host_case(wl, 0, wl.E)
+        oracle.inv_helmholtz(host["S"], host["D"], host["u"], 1)
+        t0 = time.perf_counter()
+        oracle.inv_helmholtz(host["S"], host["D"], host["u"], 1)
+        t1 = time.perf_counter() - t0
+        rows.append({"n": n, "E": wl.E, "ms": ms, "elements_per_s": wl.E / (ms * 1e-3),
+                     "gflops": wl.E * wl.flops_per_element / (ms * 1e-3) / 1e9,
+                     "oracle_1thread_ms": t1 * 1e3,
+                     "oracle_1thread_elements_per_s": wl.E / t1})
+    return rows
 
 
 def run_e2e(torch, ops, wl, case, dev, stream, steps, world, dist):
@@ -421,7 +591,7 @@ def run_e2e(torch, ops, wl, case, dev, stream, steps, world, dist):
     host_in = {k: torch.empty(case[k].shape, dtype=case[k].dtype, pin_memory=True).copy_(case[k])
                for k in names}
     out_shape = (E,) + tuple(wl.m)
-    host_out = torch.empty(out_shape, dtype=torch.float64, pin_memory=True)
+    host_out = torch.empty(out_shape, dtype=case["u"].dtype, pin_memory=True)
     mats = {k: case[k].cpu() for k in (("S",) if wl.op == "inv_helmholtz" else ("A", "B", "C"))}
     torch.cuda.synchronize(dev)
 

@@ -24,11 +24,11 @@
  *    only read; the output is fully overwritten.
  *  - Work distribution: a launch in which a CTA gets more than one batch of
  *    elements hands the batches out through a counter (16 bytes) taken from a fixed
- *    ring of 4096 inside the library image and zeroed in stream order right before the
- *    kernel (one cudaMemsetAsync on `stream`; it is captured with the kernel when
- *    the stream is being captured).  A counter comes round again after 4096
- *    launches; a kernel whose counter was touched by another launch while it ran
- *    says so through ekl_tpo_device_error_flags (bit 1).
+ *    ring of 4096 inside the library image.  The kernel itself puts the counter back
+ *    to zero when its last CTA leaves, so a call is still one kernel launch and
+ *    nothing else.  A counter comes round again after 4096 launches; a kernel whose
+ *    counter was touched by another launch while it ran says so through
+ *    ekl_tpo_device_error_flags (bit 1).
  *  - Errors: a status code is returned; nothing is thrown, aborted or trapped,
  *    and arguments that are accepted can never index out of bounds.  Validation
  *    happens before anything is enqueued:

@@ -28,7 +28,7 @@ cudaError_t launch_conv(const double* Dvq, const double* Ivq, const double* M, c
     long long grid = (long long)ekl::sm_count() * C::kCtasPerSm;
     if (grid > E) grid = E;
     unsigned long long* tickets = nullptr;
-    err = ekl::tickets_for(E, grid, stream, &tickets);
+    err = ekl::tickets_for(E, grid, &tickets);
     if (err != cudaSuccess) return err;
     ekl::dmma::convection_dmma<NQ, NV><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
         Dvq, Ivq, M, P, F, E, tickets);

@@ -82,8 +82,8 @@ bool tuned_kernels_allowed();
 // Number of SMs of the current device (cached per device).
 int sm_count();
 
-// A zeroed ticket counter (two 64-bit words) for one launch on `stream`; see launch.cu.
-cudaError_t next_ticket_counter(cudaStream_t stream, unsigned long long** out);
+// A ticket counter (two 64-bit words, zero) for one launch; see launch.cu.
+cudaError_t next_ticket_counter(unsigned long long** out);
 
 // Tensor-path kernels (fp64 arithmetic; T is the type of the fields in memory).  Return false
 // if there is no instance for these extents or the pointers do not meet the alignment the

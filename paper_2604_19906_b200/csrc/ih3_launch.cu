@@ -22,7 +22,7 @@ cudaError_t launch_ih3(const double* S0, const double* S1, const double* S2, con
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, stream, &tickets);
+    err = tickets_for(batches, grid, &tickets);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S0, S1, S2, D, u, v, E, tickets);
     return cudaGetLastError();

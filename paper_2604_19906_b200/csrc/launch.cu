@@ -25,17 +25,17 @@ int sm_count() {
 }
 
 // ---- ticket counters for the dynamic distribution of batches (BatchQueue in tpo_dmma.cuh).
-// A launch that wants one takes the next pair of 64-bit words of this ring and zeroes it in
-// stream order just before the kernel.  The ring lives in the library image (nothing is
-// allocated per call); a pair comes round again after kTicketSlots launches, and a kernel
-// whose pair was touched by another launch while it ran reports that through
-// ekl_tpo_device_error_flags (bit 1).
+// A launch that wants one takes the next pair of 64-bit words of this ring.  The ring lives in
+// the library image (nothing is allocated per call) and starts out zero; the CTA of a launch
+// that leaves last puts its pair back to zero, so no call has to clear anything.  A pair comes
+// round again after kTicketSlots launches, and a kernel whose pair was touched by another
+// launch while it ran reports that through ekl_tpo_device_error_flags (bit 1).
 namespace {
 constexpr unsigned kTicketSlots = 4096;
 __device__ unsigned long long g_ticket_ring[2 * kTicketSlots];
 }  // namespace
 
-cudaError_t next_ticket_counter(cudaStream_t stream, unsigned long long** out) {
+cudaError_t next_ticket_counter(unsigned long long** out) {
     static std::mutex mu;
     static unsigned long long* base[64] = {nullptr};
     static std::atomic<unsigned> turn{0};
@@ -54,10 +54,7 @@ cudaError_t next_ticket_counter(cudaStream_t stream, unsigned long long** out) {
         }
         b = base[dev];
     }
-    unsigned long long* slot = b + 2 * (turn.fetch_add(1, std::memory_order_relaxed) % kTicketSlots);
-    err = cudaMemsetAsync(slot, 0, 2 * sizeof(unsigned long long), stream);
-    if (err != cudaSuccess) return err;
-    *out = slot;
+    *out = b + 2 * (turn.fetch_add(1, std::memory_order_relaxed) % kTicketSlots);
     return cudaSuccess;
 }
 

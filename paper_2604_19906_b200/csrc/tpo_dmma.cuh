@@ -47,38 +47,39 @@ static inline int take_timeout_flag() {
     return flag & 3;
 }
 
-// Hands the batches of a launch to its CTAs.  Every CTA starts on batch blockIdx.x.  With a
-// ticket counter (two 64-bit words in global memory, zeroed in stream order before the launch)
-// the later batches go to whichever CTA asks first: co-resident CTAs do not get equal shares of
-// an SM, and a fixed round-robin share makes the launch wait for the slowest of them.  A CTA
-// always knows its next batch one iteration ahead (it prefetches that batch), so a ticket is
-// drawn at the top of an iteration and used two iterations later.  Without a counter
+// Hands the batches of a launch to its CTAs.  Every CTA starts on batch blockIdx.x and goes on
+// to blockIdx.x + gridDim.x.  With a ticket counter (two 64-bit words in global memory that are
+// zero when the kernel starts) the batches from 2 * gridDim.x on go to whichever CTA asks
+// first: co-resident CTAs do not get equal shares of an SM, and a fixed round-robin share
+// makes the launch wait for the slowest of them.  A CTA always knows its next batch one
+// iteration ahead (it prefetches that batch), so a ticket is drawn at the top of an iteration
+// and used two iterations later, and no CTA ever waits for the counter.  Without a counter
 // (nullptr) the batches are dealt round-robin.
 struct BatchQueue {
     unsigned long long* ticket;
     long long* shared_next;       // one value in shared memory
     long long batch, next;
     unsigned long long drawn;
+    bool handed_over;             // has publish() run yet?
 
-    // All threads; the caller synchronises the CTA before started().
     __device__ __forceinline__ void start(unsigned long long* t, long long* sh) {
         ticket = t;
         shared_next = sh;
         batch = blockIdx.x;
         next = batch + gridDim.x;
         drawn = 0;
-        if (ticket && threadIdx.x == 0) *sh = (long long)gridDim.x + (long long)atomicAdd(ticket, 1ull);
+        handed_over = false;
     }
-    __device__ __forceinline__ void started() {
-        if (ticket) next = *shared_next;
-    }
+    __device__ __forceinline__ void started() {}
     // Top of an iteration: ask for the batch after next.
     __device__ __forceinline__ void draw() {
         if (ticket && threadIdx.x == 0) drawn = atomicAdd(ticket, 1ull);
     }
     // Before a CTA barrier at or after the end of the iteration.
     __device__ __forceinline__ void publish() {
-        if (ticket && threadIdx.x == 0) *shared_next = (long long)gridDim.x + (long long)drawn;
+        if (ticket && threadIdx.x == 0)
+            *shared_next = 2ll * (long long)gridDim.x + (long long)drawn;
+        handed_over = true;
     }
     // After that barrier.
     __device__ __forceinline__ void advance() {
@@ -91,19 +92,23 @@ struct BatchQueue {
         batch = next;
         if (!ticket) next += gridDim.x;
     }
+    // (the first iteration has nothing to pick up: its next batch is the fixed one)
     __device__ __forceinline__ void refresh() {
-        if (ticket) next = *shared_next;
+        if (ticket && handed_over) next = *shared_next;
     }
     // End of the kernel: the CTA that leaves last checks that the counter holds exactly the
-    // draws of this launch (one per CTA at the start, one per batch).
+    // draws of this launch (one per batch) and leaves both words
+    // zero for the launch that gets this counter next.
     __device__ __forceinline__ void finish(long long n_batches) {
         if (ticket && threadIdx.x == 0) {
             __threadfence();
             const unsigned long long gone = atomicAdd(ticket + 1, 1ull);
             if (gone == gridDim.x - 1) {
                 const unsigned long long draws = atomicAdd(ticket, 0ull);
-                if (draws != (unsigned long long)gridDim.x + (unsigned long long)n_batches)
+                if (draws != (unsigned long long)n_batches)
                     atomicOr(&g_bulk_wait_timeout, 2);
+                atomicExch(ticket, 0ull);
+                atomicExch(ticket + 1, 0ull);
             }
         }
     }

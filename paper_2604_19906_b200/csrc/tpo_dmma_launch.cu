@@ -28,7 +28,7 @@ cudaError_t launch_ih(const T* S, const T* D, const double* lam, const double* c
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, stream, &tickets);
+    err = tickets_for(batches, grid, &tickets);
     if (err != cudaSuccess) return err;
     dmma::inv_helmholtz_dmma<N, T, LAMBDA>
         <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, lam, cvec, u, v, E, tickets);
@@ -49,7 +49,7 @@ cudaError_t launch_ih_tf32(const float* S, const float* D, const float* u, float
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, stream, &tickets);
+    err = tickets_for(batches, grid, &tickets);
     if (err != cudaSuccess) return err;
     tf32::inv_helmholtz_tf32<N>
         <<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(S, D, u, v, E, tickets);
@@ -134,7 +134,7 @@ cudaError_t launch_ap_tf32(const float* A, const float* B, const float* Cm, cons
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, stream, &tickets);
+    err = tickets_for(batches, grid, &tickets);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
     return cudaGetLastError();
@@ -182,7 +182,7 @@ cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, lon
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, stream, &tickets);
+    err = tickets_for(batches, grid, &tickets);
     if (err != cudaSuccess) return err;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
     return cudaGetLastError();

@@ -199,6 +199,24 @@ def cpu_baseline(wl, target_seconds=4.0, max_elements=None):
             }, v, ns
 
 
+def small_sets(wl) -> int:
+    """Buffer sets the cold variant of a workload that fits in L2 rotates over."""
+    return int(min(4096, max(3, -(-int(3 * L2_BYTES) // (wl.E * wl.bytes_per_element)))))
+
+
+def config_for(wl, world: int) -> dict:
+    """The `config` object of the JSON line; the same for both arms."""
+    nbytes = wl.E * wl.bytes_per_element
+    if nbytes > 2 * L2_BYTES:
+        l2 = f"inputs larger than L2 ({nbytes / 1e9:.2f} GB per step)"
+    elif world == 1 and wl.op == "inv_helmholtz" and wl.dtype == "f64":
+        l2 = f"rotating over {small_sets(wl)} buffer sets (3 x L2) between calls"
+    else:
+        l2 = "working set fits in L2 (warm)"
+    return {"workload": wl.name, "elements_per_gpu": wl.E, "l2": l2,
+            "parallelism": f"elements sharded over {world} GPU(s), no collective"}
+
+
 def reference_arm(args, wl, rank):
     """``--impl reference``: the oracle timed on the host cores, bounded sample per step."""
     if rank != 0:
@@ -232,7 +250,8 @@ def reference_arm(args, wl, rank):
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-            "config": {"workload": wl.name, "elements_per_step": ns},
+            "config": config_for(wl, int(os.environ.get("WORLD_SIZE", "1"))),
+            "sample_elements_per_step": ns,
             "gflops": value * wl.flops_per_element / 1e9,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": sample},
@@ -466,12 +485,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-            "config": {"workload": wl.name, "elements_per_gpu": E,
-                       "l2": f"inputs larger than L2 ({bytes_launch / 1e9:.2f} GB per step)"
-                       if bytes_launch > 2 * L2_BYTES else
-                       (f"rotating over {small['sets']} buffer sets (3 x L2) between calls"
-                        if small is not None and world == 1 else "working set fits in L2 (warm)"),
-                       "parallelism": f"elements sharded over {world} GPU(s), no collective"},
+            "config": config_for(wl, world),
             "gflops": value * wl.flops_per_element / 1e9,
             "roofline": roof, "clocks": clocks, "gpu_launches": args.steps,
             "max_rel_err_vs_oracle": max_rel_err}
@@ -508,7 +522,7 @@ def small_workload_variants(torch, inputs, wl, fn, dev, stream, ops, reps=200):
     n, E = wl.n[0], wl.E
     base = inputs.device_case(wl, dev)
     set_bytes = E * wl.bytes_per_element
-    sets = int(min(4096, max(3, -(-int(3 * L2_BYTES) // set_bytes))))
+    sets = small_sets(wl)
     us = [base["u"]] + [base["u"].clone() for _ in range(sets - 1)]
     Ds = [base["D"]] + [base["D"].clone() for _ in range(sets - 1)]
     vs = [torch.empty_like(base["u"]) for _ in range(sets)]

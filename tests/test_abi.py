@@ -174,3 +174,21 @@ def test_header_compiles_as_c_and_validation_answers_from_a_c_program(lib, tmp_p
     r = subprocess.run([exe], capture_output=True, text=True)
     assert r.returncode == 0, r.stdout + r.stderr
     assert "abi_check: ok" in r.stdout
+
+
+def test_probe_library_exports_what_its_header_declares():
+    """The measurement helpers live in a library of their own, not in the product library."""
+    from paper_2604_19906_b200 import build, ops, probes
+    build.build()
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "ekl_probe.h")).read(),
+                  flags=re.S)
+    names = sorted(set(re.findall(r"\b(ekl_probe_[a-z0-9_]+)\s*\(", text)))
+    assert len(names) >= 6
+    plib = probes.library()
+    for n in names:
+        assert hasattr(plib, n), n
+        assert not hasattr(ops.library(), n), f"{n} must not be exported by the product library"
+    # argument checks answer without a GPU
+    f = ctypes.c_double(0.0)
+    assert plib.ekl_probe_fp64_fma_chain(None, 1, 1, ctypes.byref(f), None) == 1
+    assert plib.ekl_probe_fp64_dmma(ctypes.c_void_p(P), 1, 1, 3, ctypes.byref(f), None) == 2

@@ -290,7 +290,7 @@ inv_helmholtz_umma(const float* __restrict__ S, const float* __restrict__ D, con
         // not expected: flag it, then give what may still be in flight (the bulk copy into the
         // landing buffer, tensor instructions) one more bounded wait before the CTA lets go of
         // its shared and tensor memory
-        dmma::g_bulk_wait_timeout = 1;
+        atomicOr(&dmma::g_bulk_wait_timeout, 1);
         dmma::mbar_wait(bar_u, par_u);
         dmma::mbar_wait(bar_mma, par_mma);
     }

@@ -70,7 +70,6 @@ struct BatchQueue {
         drawn = 0;
         handed_over = false;
     }
-    __device__ __forceinline__ void started() {}
     // Top of an iteration: ask for the batch after next.
     __device__ __forceinline__ void draw() {
         if (ticket && threadIdx.x == 0) drawn = atomicAdd(ticket, 1ull);
@@ -552,7 +551,6 @@ inv_helmholtz_dmma(const T* __restrict__ S, const T* __restrict__ D,
     q.start(tickets, &shared_next);
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
-    q.started();
 
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
@@ -707,7 +705,6 @@ inv_helmholtz3_dmma(const double* __restrict__ S0, const double* __restrict__ S1
     q.start(tickets, &shared_next);
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
-    q.started();
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);

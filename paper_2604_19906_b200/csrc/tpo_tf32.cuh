@@ -248,7 +248,6 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
     q.start(tickets, &shared_next);
     if (threadIdx.x == 0) dmma::mbar_init(bar, 1);
     __syncthreads();
-    q.started();
     auto batch_count = [&](long long b) {
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);

@@ -127,8 +127,10 @@ ekl_tpo_status ekl_tpo_inv_helmholtz3(const double* S0, const double* S1, const 
  *   A [m0,n0]  B [m1,n1]  C [m2,n2]     u [E,n0,n1,n2]     v [E,m0,m1,m2]
  *
  * fp64.  v must not overlap any input.  Cubic shapes n -> m (n0=n1=n2, m0=m1=m2) with even
- * n, m from 4 to 16 and a 16-byte aligned u run on the FP64 tensor path; every other shape
- * that fits in shared memory runs on the general kernel.
+ * n, m from 4 to 16, and the non-cubic shapes (8,8,8)->(12,12,8), (8,8,8)->(8,8,12),
+ * (12,12,12)->(8,8,12), (12,12,8)->(8,8,12), (8,10,12)->(12,10,8), (8,10,12)->(8,10,12),
+ * (6,8,10)->(10,8,6), (14,12,8)->(8,12,14), with a 16-byte aligned u run on the FP64 tensor
+ * path; every other shape that fits in shared memory runs on the general kernel.
  */
 ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
                              const double* u, double* v,

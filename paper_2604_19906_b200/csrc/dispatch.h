@@ -75,6 +75,7 @@ cudaError_t launch_convection_generic(const double* Dvq, const double* Ivq, cons
 // Helmholtz kernels (see ekl_tpo_device_error_flags).
 int convection_timeout_flag();
 int ih3_timeout_flag();
+int apply_aniso_timeout_flag();
 
 // False when EKL_TPO_VARIANT=generic asks for the run-time-sized kernels only.
 bool tuned_kernels_allowed();
@@ -99,6 +100,10 @@ bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double*
 bool try_launch_ih3_dmma(const double* S0, const double* S1, const double* S2, const double* D,
                          const double* u, double* v, int n0, int n1, int n2, long long E,
                          cudaStream_t stream, cudaError_t* err);
+// Forward operator, shapes that are not cubic (fp64).
+bool try_launch_apply_aniso(const double* A, const double* B, const double* C, const double* u,
+                            double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
+                            cudaStream_t stream, cudaError_t* err);
 template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,

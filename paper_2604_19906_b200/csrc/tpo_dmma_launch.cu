@@ -276,7 +276,16 @@ bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v,
                            cudaError_t* err) {
     // fp64 u is bulk-copied plane by plane: 16-byte aligned element addresses
     if (sizeof(T) == 8 && reinterpret_cast<uintptr_t>(u) % 16) return false;
-    if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) return false;
+    if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) {
+        if constexpr (sizeof(T) == 8)
+            return try_launch_apply_aniso(reinterpret_cast<const double*>(A),
+                                          reinterpret_cast<const double*>(B),
+                                          reinterpret_cast<const double*>(C),
+                                          reinterpret_cast<const double*>(u),
+                                          reinterpret_cast<double*>(v), n0, n1, n2, m0, m1, m2, E,
+                                          stream, err);
+        return false;
+    }
     if (try_launch_apply_tf32(A, B, C, u, v, n0, m0, E, stream, err)) return true;
     switch (n0) {
         case 4: return apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err);
@@ -334,7 +343,7 @@ extern "C" ekl_tpo_status ekl_tpo_selftest_expired_wait(cudaStream_t stream) {
 extern "C" int ekl_tpo_device_error_flags(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return -1;
     const int a = ekl::dmma::take_timeout_flag(), b = ekl::convection_timeout_flag(),
-              c = ekl::ih3_timeout_flag();
-    if (a < 0 || b < 0 || c < 0) return -1;
-    return a | b | c;
+              c = ekl::ih3_timeout_flag(), d = ekl::apply_aniso_timeout_flag();
+    if (a < 0 || b < 0 || c < 0 || d < 0) return -1;
+    return a | b | c | d;
 }

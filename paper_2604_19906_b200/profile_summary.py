@@ -5,7 +5,7 @@ records the DRAM traffic per element that ``bench.py`` prints as ``roofline.traf
         [--workload KEY --elements E]      # also update profiles/dram_traffic.json
         [--out profiles/NAME.md --command "the command that produced the report"]
 
-The JSON entry stores, beside the bytes per element, a digest of the kernel sources at the
+The JSON entry stores, beside the bytes per element, a digest of the kernel sources (csrc/*.cuh) at the
 time of the capture; ``bench.py`` reports ``traffic: null`` once the sources have changed.
 ``ncu`` must be on PATH (it reads reports without a GPU).
 """
@@ -50,9 +50,10 @@ METRICS = [
 
 
 def source_digest() -> str:
-    """SHA-256 over the kernel sources (every file under csrc/), in name order."""
+    """SHA-256 over the kernel sources (the .cuh files under csrc/, where every kernel and its
+    launch configuration live; the .cu files only select and launch), in name order."""
     h = hashlib.sha256()
-    for path in sorted(glob.glob(os.path.join(PKG, "csrc", "*"))):
+    for path in sorted(glob.glob(os.path.join(PKG, "csrc", "*.cuh"))):
         h.update(os.path.basename(path).encode())
         with open(path, "rb") as f:
             h.update(f.read())

@@ -279,6 +279,33 @@ def test_apply_f64_cubic_pairs_on_the_tensor_path(env, n, m, E):
     assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
 
 
+ANISO = [((8, 8, 8), (12, 12, 8)), ((8, 8, 8), (8, 8, 12)), ((12, 12, 12), (8, 8, 12)),
+         ((12, 12, 8), (8, 8, 12)), ((8, 10, 12), (12, 10, 8)), ((8, 10, 12), (8, 10, 12)),
+         ((6, 8, 10), (10, 8, 6)), ((14, 12, 8), (8, 12, 14))]
+
+
+@pytest.mark.parametrize("nn,mm", ANISO)
+@pytest.mark.parametrize("E", [1, 2, 3, 257, 4001])
+def test_apply_f64_non_cubic_shapes_on_the_tensor_path(env, nn, mm, E):
+    """Three different operators on all-distinct extents: any axis mix-up fails.  E = 4001 gives
+    every CTA several batches (the dynamic deal of batches)."""
+    g = rng(hash((nn, mm)) % 9973 + E)
+    A, B, C = (g.standard_normal((mm[d], nn[d])) / np.sqrt(nn[d]) for d in range(3))
+    u = g.uniform(-1, 1, (E,) + nn)
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    v = env["torch"].full((E,) + mm, float("nan"), dtype=env["torch"].float64, device=env["dev"])
+    got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C, u)), out=v)
+    env["torch"].cuda.synchronize()
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+    # the same shape through the general kernel (an unaligned u falls back to it) agrees
+    if E == 257:
+        buf = env["torch"].zeros(u.size + 1, dtype=env["torch"].float64, device=env["dev"])
+        uu = buf[1:].view(u.shape)
+        uu.copy_(to_dev(env, u))
+        got2 = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C)), uu)
+        assert env["oracle"].rel_err_per_element(got2.cpu().numpy(), want).max() <= TOL64
+
+
 @pytest.mark.parametrize("nn,mm", SHAPES[:3])
 def test_apply_f32(env, nn, mm):
     g = rng(3)

@@ -126,11 +126,14 @@ ekl_tpo_status ekl_tpo_inv_helmholtz3(const double* S0, const double* S1, const 
  *
  *   A [m0,n0]  B [m1,n1]  C [m2,n2]     u [E,n0,n1,n2]     v [E,m0,m1,m2]
  *
- * fp64.  v must not overlap any input.  Cubic shapes n -> m (n0=n1=n2, m0=m1=m2) with even
- * n, m from 4 to 16, and the non-cubic shapes (8,8,8)->(12,12,8), (8,8,8)->(8,8,12),
+ * fp64.  v must not overlap any input.  On the FP64 tensor path run: cubic shapes n -> m
+ * (n0=n1=n2, m0=m1=m2) with even n, m from 4 to 16; the cubic shapes with an odd extent
+ * n -> n for odd n from 5 to 15, n <-> n+2 for odd n from 5 to 13, n <-> n+1 for n from 4 to 9,
+ * and 5 <-> 8, 6 <-> 9, 7 <-> 11, 9 <-> 14, 10 <-> 15 (to and from the 3/2 quadrature
+ * resolution); and the non-cubic shapes (8,8,8)->(12,12,8), (8,8,8)->(8,8,12),
  * (12,12,12)->(8,8,12), (12,12,8)->(8,8,12), (8,10,12)->(12,10,8), (8,10,12)->(8,10,12),
- * (6,8,10)->(10,8,6), (14,12,8)->(8,12,14), with a 16-byte aligned u run on the FP64 tensor
- * path; every other shape that fits in shared memory runs on the general kernel.
+ * (6,8,10)->(10,8,6), (14,12,8)->(8,12,14).  Where n1*n2 is even, u must be 16-byte aligned
+ * for that path.  Every other case that fits in shared memory runs on the general kernel.
  */
 ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
                              const double* u, double* v,
@@ -153,7 +156,8 @@ ekl_tpo_status ekl_tpo_apply(const double* A, const double* B, const double* C,
  * in this header, so the differentiation matrix acts on the fastest axis for direction 0, on
  * the middle one for direction 1 and on the slowest for direction 2.  fp64.  F must not
  * overlap any input.  (nq,nv) in {(4,4),(6,4),(6,6),(8,4),(8,6),(8,8),(10,8),(10,10),(12,8),
- * (12,10),(12,12),(14,12)} with 16-byte aligned M and P run on the FP64 tensor path; every
+ * (12,10),(12,12),(14,12)} and {(5,5),(7,5),(7,7),(8,5),(9,6),(9,7),(9,9),(11,7),(14,9),
+ * (15,10)} run on the FP64 tensor path (M and P 16-byte aligned where nq is even); every
  * other combination that fits in shared memory (nq, nv <= 64 and about 2 max(nq,nv)^3 + nv^3
  * values) runs on a general kernel; larger extents return EKL_TPO_ERR_UNSUPPORTED.
  */
@@ -168,7 +172,8 @@ ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Ivq, const do
  * 16-byte aligned u, run on the TF32 tensor path with split operands: every
  * product is taken as a_hi*b_hi + a_lo*b_hi + a_hi*b_lo (hi = the value rounded to TF32, lo =
  * the rest) and accumulated in fp32, the fields stay fp32 on chip; measured error about 4e-7.
- * On the FP64 tensor path (the other extents from 4 to 20, the other cubic pairs) the fields
+ * On the FP64 tensor path (the other extents from 4 to 20, the other cubic pairs listed for
+ * ekl_tpo_apply) the fields
  * are widened to fp64 on chip, all arithmetic is fp64, and v is rounded to fp32 once when it
  * is stored; the general kernel computes in fp32.  With EKL_TPO_F32_PATH=tcgen05 in the
  * environment (read once, at the first call) the split-TF32 case runs on tcgen05.mma with the

@@ -38,7 +38,9 @@ struct ConvCfg {
     static constexpr size_t kSmemBytes = (size_t)kDoubles * sizeof(double) + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
     static constexpr int kCtasPerSm = kBySmem < 1 ? 1 : (kBySmem > 2 ? 2 : kBySmem);
-    static_assert(NQ % 2 == 0 && NV % 2 == 0, "even extents (bulk copies, paired stores)");
+    // bulk copies need planes that are whole 16-byte units; an odd nq uses 8-byte asynchronous
+    // copies issued by all threads
+    static constexpr bool kBulk = (NQ % 2 == 0);
     static_assert(S1::kMTiles == S2::kMTiles && S1::kKSteps == S3::kKSteps, "one fragment shape");
 };
 
@@ -72,15 +74,31 @@ __device__ __forceinline__ void tile_store(const double (&c)[SS::kMTiles][2], do
                                            int lane) {
     const int r = lane >> 2, kk = lane & 3;
     const int qs = 8 * t + 2 * kk;
-    if (qs >= SS::kPencils) return;
-    const int ps1 = qs / SS::E2;
-    double* dst = out + ps1 * SS::OUT_PS + (qs - ps1 * SS::E2) * SS::OUT_RS;
+    if constexpr (SS::kPaired) {
+        // even rows: the two pencils of a lane share a row, one address serves both
+        if (qs >= SS::kPencils) return;
+        const int ps1 = qs / SS::E2;
+        double* dst = out + ps1 * SS::OUT_PS + (qs - ps1 * SS::E2) * SS::OUT_RS;
 #pragma unroll
-    for (int mt = 0; mt < SS::kMTiles; ++mt) {
-        const int o = 8 * mt + r;
-        if (o < SS::O) {
-            dst[o] = c[mt][0];
-            dst[SS::OUT_RS + o] = c[mt][1];
+        for (int mt = 0; mt < SS::kMTiles; ++mt) {
+            const int o = 8 * mt + r;
+            if (o < SS::O) {
+                dst[o] = c[mt][0];
+                dst[SS::OUT_RS + o] = c[mt][1];
+            }
+        }
+    } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int q = qs + h;
+            if (q >= SS::kPencils) continue;
+            const int ps1 = q / SS::E2;
+            double* dst = out + ps1 * SS::OUT_PS + (q - ps1 * SS::E2) * SS::OUT_RS;
+#pragma unroll
+            for (int mt = 0; mt < SS::kMTiles; ++mt) {
+                const int o = 8 * mt + r;
+                if (o < SS::O) dst[o] = c[mt][h];
+            }
         }
     }
 }
@@ -131,8 +149,21 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
                           (unsigned)(NQ * NQ * sizeof(double)), bar);
         }
     };
+    // all threads: the same transfer by 8-byte asynchronous copies, for fields whose planes are
+    // not a whole number of 16-byte units (odd nq)
+    auto fetch_copy = [&](int c, long long e, bool with_m) {
+        if (with_m)
+            copy_elements<NQ, NQ * NQ, C::kPS0, C::kES0, double>(sM, M + (size_t)e * kQ3, 1);
+        for (int d = 0; d < 3; ++d)
+            copy_elements<NQ, NQ * NQ, C::kPS0, C::kES0, double>(
+                sX + d * C::kES0, P + (((size_t)c * 3 + d) * E + e) * kQ3, 1);
+    };
 
-    if (threadIdx.x == 0 && q.batch < E) fetch(0, q.batch, true);
+    if constexpr (C::kBulk) {
+        if (threadIdx.x == 0 && q.batch < E) fetch(0, q.batch, true);
+    } else {
+        if (q.batch < E) fetch_copy(0, q.batch, true);
+    }
     unsigned parity = 0;
     bool ok = true;
     while (ok && q.batch < E) {
@@ -145,11 +176,15 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             for (int cd = 3; cd < 9; ++cd) bulk_prefetch_l2(P + ((size_t)cd * E + e) * kQ3, field);
         }
         for (int c = 0; c < 3; ++c) {
-            if (!wait_bulk(bar, parity)) {
-                ok = false;
-                break;
+            if constexpr (C::kBulk) {
+                if (!wait_bulk(bar, parity)) {
+                    ok = false;
+                    break;
+                }
+                parity ^= 1u;
+            } else {
+                wait_copies();
             }
-            parity ^= 1u;
             if (c == 0) {
                 // the barrier inside the wait orders the ticket handed over at the end of the
                 // previous element; now the next element is known: ask L2 for its first fields
@@ -176,13 +211,19 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             }
             __syncthreads();
             // the P buffers (and, after the last component, M) are free: fetch what comes next
-            if (threadIdx.x == 0) {
+            if constexpr (C::kBulk) {
+                if (threadIdx.x == 0) {
+                    const bool last = (c == 2);
+                    const long long ne = last ? q.next : e;
+                    if (ne < E) {
+                        fence_async_proxy();
+                        fetch(last ? 0 : c + 1, ne, last);
+                    }
+                }
+            } else {
                 const bool last = (c == 2);
                 const long long ne = last ? q.next : e;
-                if (ne < E) {
-                    fence_async_proxy();
-                    fetch(last ? 0 : c + 1, ne, last);
-                }
+                if (ne < E) fetch_copy(last ? 0 : c + 1, ne, last);
             }
             // stage 2: w0 = I t0 (first kTiles tasks), w12 = D t1 + I t2 (the rest)
 #pragma unroll

@@ -3,37 +3,10 @@
 
 #include <cstdint>
 
-#include "convection_dmma.cuh"
+#include "convection_launch.h"
 #include "dispatch.h"
-#include "launch_util.h"
 
 namespace {
-
-template <int NQ, int NV>
-cudaError_t launch_conv(const double* Dvq, const double* Ivq, const double* M, const double* P,
-                        double* F, long long E, cudaStream_t stream) {
-    using C = ekl::dmma::ConvCfg<NQ, NV>;
-    static_assert(C::kSmemBytes <= ekl::kMaxSmemBytes, "instance does not fit in shared memory");
-    static bool prepared[64] = {false};
-    int dev = 0;
-    cudaError_t err = cudaGetDevice(&dev);
-    if (err != cudaSuccess) return err;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!prepared[dev]) {
-        err = cudaFuncSetAttribute(ekl::dmma::convection_dmma<NQ, NV>,
-                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
-        if (err != cudaSuccess) return err;
-        prepared[dev] = true;
-    }
-    long long grid = (long long)ekl::sm_count() * C::kCtasPerSm;
-    if (grid > E) grid = E;
-    unsigned long long* tickets = nullptr;
-    err = ekl::tickets_for(E, grid, &tickets);
-    if (err != cudaSuccess) return err;
-    ekl::dmma::convection_dmma<NQ, NV><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
-        Dvq, Ivq, M, P, F, E, tickets);
-    return cudaGetLastError();
-}
 
 bool misaligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
@@ -59,8 +32,9 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
     if (misaligned(Dvq, 8) || misaligned(Ivq, 8) || misaligned(F, 8) || misaligned(M, 8) ||
         misaligned(P, 8))
         return EKL_TPO_ERR_ALIGN;
-    // the tensor-path instances bulk-copy M and P: 16-byte aligned fields
-    const bool tensor_ok = ekl::tuned_kernels_allowed() && !misaligned(M, 16) && !misaligned(P, 16);
+    // the tensor-path instances bulk-copy M and P where nq is even: 16-byte aligned fields
+    const bool tensor_ok = ekl::tuned_kernels_allowed() &&
+                           (nq % 2 != 0 || (!misaligned(M, 16) && !misaligned(P, 16)));
     const size_t q3 = (size_t)nq * nq * nq * sizeof(double), v3 = (size_t)nv * nv * nv * sizeof(double);
     const size_t fbytes = 3 * (size_t)E * v3, mat = (size_t)nv * nq * sizeof(double);
     if (overlaps(F, fbytes, M, (size_t)E * q3) || overlaps(F, fbytes, P, 9 * (size_t)E * q3) ||
@@ -69,7 +43,7 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
     cudaError_t err = cudaSuccess;
 #define EKL_CONV_CASE(Q, V)                                                   \
     if (tensor_ok && nq == Q && nv == V) {                                    \
-        err = launch_conv<Q, V>(Dvq, Ivq, M, P, F, E, stream);                \
+        err = ekl::launch_conv<Q, V>(Dvq, Ivq, M, P, F, E, stream);                \
         if (err != cudaSuccess) {                                             \
             ekl::set_last_cuda_error((int)err);                               \
             return EKL_TPO_ERR_CUDA;                                          \
@@ -89,6 +63,13 @@ extern "C" ekl_tpo_status ekl_tpo_convection(const double* Dvq, const double* Iv
     EKL_CONV_CASE(12, 12)
     EKL_CONV_CASE(14, 12)
 #undef EKL_CONV_CASE
+    if (tensor_ok && ekl::try_launch_convection_odd(Dvq, Ivq, M, P, F, nq, nv, E, stream, &err)) {
+        if (err != cudaSuccess) {
+            ekl::set_last_cuda_error((int)err);
+            return EKL_TPO_ERR_CUDA;
+        }
+        return EKL_TPO_OK;
+    }
     err = ekl::launch_convection_generic(Dvq, Ivq, M, P, F, nq, nv, E, stream);
     if (err != cudaSuccess) {
         ekl::set_last_cuda_error((int)err);

@@ -1,0 +1,36 @@
+// Launch of one convective-flux instance on the FP64 tensor path; shared by the translation
+// units that hold the instances.
+#pragma once
+#include "convection_dmma.cuh"
+#include "dispatch.h"
+#include "launch_util.h"
+
+namespace ekl {
+
+template <int NQ, int NV>
+cudaError_t launch_conv(const double* Dvq, const double* Ivq, const double* M, const double* P,
+                        double* F, long long E, cudaStream_t stream) {
+    using C = dmma::ConvCfg<NQ, NV>;
+    static_assert(C::kSmemBytes <= kMaxSmemBytes, "instance does not fit in shared memory");
+    static bool prepared[64] = {false};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!prepared[dev]) {
+        err = cudaFuncSetAttribute(dmma::convection_dmma<NQ, NV>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+        if (err != cudaSuccess) return err;
+        prepared[dev] = true;
+    }
+    long long grid = (long long)sm_count() * C::kCtasPerSm;
+    if (grid > E) grid = E;
+    unsigned long long* tickets = nullptr;
+    err = tickets_for(E, grid, &tickets);
+    if (err != cudaSuccess) return err;
+    dmma::convection_dmma<NQ, NV><<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(
+        Dvq, Ivq, M, P, F, E, tickets);
+    return cudaGetLastError();
+}
+
+}  // namespace ekl

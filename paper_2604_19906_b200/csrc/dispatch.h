@@ -71,11 +71,20 @@ cudaError_t launch_convection_generic(const double* Dvq, const double* Ivq, cons
                                       const double* P, double* F, int nq, int nv, long long E,
                                       cudaStream_t stream);
 
+// Convective-flux instances with an odd extent; false if there is none for (nq, nv).
+bool try_launch_convection_odd(const double* Dvq, const double* Ivq, const double* M,
+                               const double* P, double* F, int nq, int nv, long long E,
+                               cudaStream_t stream, cudaError_t* err);
+
 // Device error flags of the convective-flux kernels and of the per-direction inverse
 // Helmholtz kernels (see ekl_tpo_device_error_flags).
 int convection_timeout_flag();
+int convection_odd_timeout_flag();
 int ih3_timeout_flag();
 int apply_aniso_timeout_flag();
+int apply_odd_a_timeout_flag();
+int apply_odd_b_timeout_flag();
+int apply_odd_c_timeout_flag();
 
 // False when EKL_TPO_VARIANT=generic asks for the run-time-sized kernels only.
 bool tuned_kernels_allowed();
@@ -104,6 +113,17 @@ bool try_launch_ih3_dmma(const double* S0, const double* S1, const double* S2, c
 bool try_launch_apply_aniso(const double* A, const double* B, const double* C, const double* u,
                             double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
                             cudaStream_t stream, cudaError_t* err);
+// Forward operator, cubic n -> m with an odd extent (three groups of instances, one translation
+// unit each).
+template <typename T>
+bool try_launch_apply_odd_a(const T* A, const T* B, const T* C, const T* u, T* v, int n, int m,
+                            long long E, cudaStream_t stream, cudaError_t* err);
+template <typename T>
+bool try_launch_apply_odd_b(const T* A, const T* B, const T* C, const T* u, T* v, int n, int m,
+                            long long E, cudaStream_t stream, cudaError_t* err);
+template <typename T>
+bool try_launch_apply_odd_c(const T* A, const T* B, const T* C, const T* u, T* v, int n, int m,
+                            long long E, cudaStream_t stream, cudaError_t* err);
 template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,

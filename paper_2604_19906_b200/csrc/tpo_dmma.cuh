@@ -792,7 +792,8 @@ struct ApplyCfg {
     static constexpr int kByWarps = 20 / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
-    static_assert((N1 * N2) % 2 == 0, "planes must be a whole number of 16-byte units");
+    // bulk copies need planes that are whole 16-byte units; odd planes use 8-byte asynchronous copies
+    static constexpr bool kBulkPlanes = (N1 * N2) % 2 == 0;
 };
 
 // v[e] = (A(x)B(x)C) u[e]; contraction order A, B, C (slowest axis first).
@@ -802,7 +803,7 @@ __global__ void __launch_bounds__(ApplyCfg<N0, N1, N2, M0, M1, M2>::kThreads,
 apply_dmma(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict__ Cm,
            const T* __restrict__ u, T* __restrict__ v, long long E, unsigned long long* tickets) {
     using C = ApplyCfg<N0, N1, N2, M0, M1, M2>;
-    constexpr bool kBulk = sizeof(T) == sizeof(double);
+    constexpr bool kBulk = sizeof(T) == sizeof(double) && C::kBulkPlanes;
     using S1 = typename C::S1;
     using S2 = typename C::S2;
     using S3 = typename C::S3;

@@ -8,6 +8,7 @@
 #include "tpo_dmma.cuh"
 #include "tpo_tf32.cuh"
 #include "tpo_umma.cuh"
+#include "apply_launch.h"
 
 #include <cstdlib>
 #include <cstring>
@@ -169,25 +170,6 @@ bool try_launch_apply_tf32(const double*, const double*, const double*, const do
     return false;
 }
 
-template <int N0, int N1, int N2, int M0, int M1, int M2, typename T>
-cudaError_t launch_ap(const T* A, const T* B, const T* Cm, const T* u, T* v, long long E,
-                      cudaStream_t stream) {
-    using C = dmma::ApplyCfg<N0, N1, N2, M0, M1, M2>;
-    auto kernel = dmma::apply_dmma<N0, N1, N2, M0, M1, M2, T>;
-    static std::atomic<int> cached[64];
-    int per_sm = 1;
-    cudaError_t err = ctas_per_sm(kernel, C::kThreads, C::kSmemBytes, cached, &per_sm);
-    if (err != cudaSuccess) return err;
-    const long long batches = (E + C::kBe - 1) / C::kBe;
-    long long grid = (long long)sm_count() * per_sm;
-    if (grid > batches) grid = batches;
-    unsigned long long* tickets = nullptr;
-    err = tickets_for(batches, grid, &tickets);
-    if (err != cudaSuccess) return err;
-    kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
-    return cudaGetLastError();
-}
-
 }  // namespace
 
 template <typename T>
@@ -226,13 +208,13 @@ template <int N, typename T>
 bool apply_cubic_from(int m, const T* A, const T* B, const T* C, const T* u, T* v, long long E,
                       cudaStream_t stream, cudaError_t* err) {
     switch (m) {
-        case 4: *err = launch_ap<N, N, N, 4, 4, 4, T>(A, B, C, u, v, E, stream); return true;
-        case 6: *err = launch_ap<N, N, N, 6, 6, 6, T>(A, B, C, u, v, E, stream); return true;
-        case 8: *err = launch_ap<N, N, N, 8, 8, 8, T>(A, B, C, u, v, E, stream); return true;
-        case 10: *err = launch_ap<N, N, N, 10, 10, 10, T>(A, B, C, u, v, E, stream); return true;
-        case 12: *err = launch_ap<N, N, N, 12, 12, 12, T>(A, B, C, u, v, E, stream); return true;
-        case 14: *err = launch_ap<N, N, N, 14, 14, 14, T>(A, B, C, u, v, E, stream); return true;
-        case 16: *err = launch_ap<N, N, N, 16, 16, 16, T>(A, B, C, u, v, E, stream); return true;
+        case 4: *err = launch_apply_instance<N, N, N, 4, 4, 4, T>(A, B, C, u, v, E, stream); return true;
+        case 6: *err = launch_apply_instance<N, N, N, 6, 6, 6, T>(A, B, C, u, v, E, stream); return true;
+        case 8: *err = launch_apply_instance<N, N, N, 8, 8, 8, T>(A, B, C, u, v, E, stream); return true;
+        case 10: *err = launch_apply_instance<N, N, N, 10, 10, 10, T>(A, B, C, u, v, E, stream); return true;
+        case 12: *err = launch_apply_instance<N, N, N, 12, 12, 12, T>(A, B, C, u, v, E, stream); return true;
+        case 14: *err = launch_apply_instance<N, N, N, 14, 14, 14, T>(A, B, C, u, v, E, stream); return true;
+        case 16: *err = launch_apply_instance<N, N, N, 16, 16, 16, T>(A, B, C, u, v, E, stream); return true;
         default: return false;
     }
 }
@@ -274,8 +256,9 @@ template <typename T>
 bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,
                            cudaError_t* err) {
-    // fp64 u is bulk-copied plane by plane: 16-byte aligned element addresses
-    if (sizeof(T) == 8 && reinterpret_cast<uintptr_t>(u) % 16) return false;
+    // fp64 u is bulk-copied plane by plane where a plane is a whole number of 16-byte units:
+    // 16-byte aligned element addresses
+    if (sizeof(T) == 8 && (n1 * n2) % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
     if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) {
         if constexpr (sizeof(T) == 8)
             return try_launch_apply_aniso(reinterpret_cast<const double*>(A),
@@ -288,15 +271,18 @@ bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v,
     }
     if (try_launch_apply_tf32(A, B, C, u, v, n0, m0, E, stream, err)) return true;
     switch (n0) {
-        case 4: return apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err);
-        case 6: return apply_cubic_from<6, T>(m0, A, B, C, u, v, E, stream, err);
-        case 8: return apply_cubic_from<8, T>(m0, A, B, C, u, v, E, stream, err);
-        case 10: return apply_cubic_from<10, T>(m0, A, B, C, u, v, E, stream, err);
-        case 12: return apply_cubic_from<12, T>(m0, A, B, C, u, v, E, stream, err);
-        case 14: return apply_cubic_from<14, T>(m0, A, B, C, u, v, E, stream, err);
-        case 16: return apply_cubic_from<16, T>(m0, A, B, C, u, v, E, stream, err);
-        default: return false;
+        case 4: if (apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 6: if (apply_cubic_from<6, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 8: if (apply_cubic_from<8, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 10: if (apply_cubic_from<10, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 12: if (apply_cubic_from<12, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 14: if (apply_cubic_from<14, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        case 16: if (apply_cubic_from<16, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
+        default: break;
     }
+    return try_launch_apply_odd_a(A, B, C, u, v, n0, m0, E, stream, err) ||
+           try_launch_apply_odd_b(A, B, C, u, v, n0, m0, E, stream, err) ||
+           try_launch_apply_odd_c(A, B, C, u, v, n0, m0, E, stream, err);
 }
 
 template bool try_launch_ih_dmma<double>(const double*, const double*, const double*, double*, int,
@@ -342,8 +328,14 @@ extern "C" ekl_tpo_status ekl_tpo_selftest_expired_wait(cudaStream_t stream) {
 // valid.  Synchronises the device.
 extern "C" int ekl_tpo_device_error_flags(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-    const int a = ekl::dmma::take_timeout_flag(), b = ekl::convection_timeout_flag(),
-              c = ekl::ih3_timeout_flag(), d = ekl::apply_aniso_timeout_flag();
-    if (a < 0 || b < 0 || c < 0 || d < 0) return -1;
-    return a | b | c | d;
+    const int flags[] = {ekl::dmma::take_timeout_flag(),   ekl::convection_timeout_flag(),
+                         ekl::ih3_timeout_flag(),          ekl::apply_aniso_timeout_flag(),
+                         ekl::apply_odd_a_timeout_flag(),  ekl::apply_odd_b_timeout_flag(),
+                         ekl::apply_odd_c_timeout_flag(),    ekl::convection_odd_timeout_flag()};
+    int all = 0;
+    for (int f : flags) {
+        if (f < 0) return -1;
+        all |= f;
+    }
+    return all;
 }

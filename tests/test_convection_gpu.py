@@ -7,6 +7,8 @@ pytestmark = pytest.mark.gpu
 TOL64 = 1e-12
 PAIRS = [(4, 4), (6, 4), (6, 6), (8, 4), (8, 6), (8, 8), (10, 8), (10, 10), (12, 8), (12, 10),
          (12, 12), (14, 12)]
+# tensor-path instances with an odd extent (odd nq: no bulk copies; odd nv: unpaired stores)
+ODD_PAIRS = [(5, 5), (7, 5), (7, 7), (8, 5), (9, 6), (9, 7), (9, 9), (11, 7), (14, 9), (15, 10)]
 
 
 @pytest.fixture(scope="module")
@@ -25,6 +27,29 @@ def case(nq, nv, E, seed):
     M = g.uniform(0.5, 1.5, (E, nq, nq, nq))
     P = g.uniform(-1, 1, (3, 3, E, nq, nq, nq))
     return Dvq, Ivq, M, P
+
+
+@pytest.mark.parametrize("nq,nv", ODD_PAIRS)
+@pytest.mark.parametrize("E", [1, 2, 5, 311, 1301])
+def test_convection_odd_extents_match_oracle(env, nq, nv, E):
+    """E = 1301 gives every CTA more than four elements (the dynamic deal); for an odd nq the
+    fields M and P also start 8 bytes off a 16-byte boundary."""
+    torch = env["torch"]
+    Dvq, Ivq, M, P = case(nq, nv, E, 100 * nq + nv + E)
+    want = env["oracle"].convection(Dvq, Ivq, M, P)
+    dev = [torch.from_numpy(np.ascontiguousarray(x)).to(env["dev"]) for x in (Dvq, Ivq, M, P)]
+    if nq % 2 == 1:
+        for i in (2, 3):
+            buf = torch.zeros(dev[i].numel() + 1, dtype=torch.float64, device=env["dev"])
+            shifted = buf[1:].view(dev[i].shape)
+            shifted.copy_(dev[i])
+            dev[i] = shifted
+    got = env["ops"].ekl_tpo_convection(*dev)
+    torch.cuda.synchronize()
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().reshape(3 * E, nv, nv, nv),
+                                            want.reshape(3 * E, nv, nv, nv))
+    assert err.max() <= TOL64, (nq, nv, E, err.max())
+    assert env["ops"].library().ekl_tpo_device_error_flags() == 0
 
 
 @pytest.mark.parametrize("nq,nv", PAIRS)
@@ -80,7 +105,7 @@ def test_convection_repeatable_guards_and_errors(env):
     assert lib.ekl_tpo_device_error_flags() == 0
 
 
-@pytest.mark.parametrize("nq,nv", [(3, 2), (5, 7), (7, 5), (9, 9), (13, 8), (16, 12), (2, 1), (1, 1)])
+@pytest.mark.parametrize("nq,nv", [(3, 2), (5, 7), (6, 5), (11, 11), (13, 8), (16, 12), (2, 1), (1, 1)])
 @pytest.mark.parametrize("E", [1, 4, 97])
 def test_convection_general_kernel_shapes(env, nq, nv, E):
     """Extents without a tensor-path instance run on the run-time-sized kernel."""

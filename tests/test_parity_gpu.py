@@ -306,6 +306,44 @@ def test_apply_f64_non_cubic_shapes_on_the_tensor_path(env, nn, mm, E):
         assert env["oracle"].rel_err_per_element(got2.cpu().numpy(), want).max() <= TOL64
 
 
+ODD_CUBIC = [(5, 5), (7, 7), (9, 9), (11, 11), (13, 13), (15, 15), (5, 7), (7, 5), (7, 9), (9, 7),
+             (9, 11), (11, 9), (11, 13), (13, 11), (13, 15), (15, 13), (5, 8), (8, 5), (6, 9), (9, 6),
+             (7, 11), (11, 7), (9, 14), (14, 9), (10, 15), (15, 10), (4, 5), (5, 4), (5, 6), (6, 5),
+             (6, 7), (7, 6), (7, 8), (8, 7), (8, 9), (9, 8), (9, 10), (10, 9)]
+
+
+@pytest.mark.parametrize("n,m", ODD_CUBIC)
+def test_apply_cubic_shapes_with_an_odd_extent(env, n, m):
+    """Cubic n -> m forward operators where n or m is odd (tensor-path instances whose fields
+    have odd planes or odd rows): three different matrices, element counts that leave a partly
+    filled batch and that give every CTA several batches, fp64 and fp32 fields, and u starting
+    8 bytes off a 16-byte boundary (allowed when a plane of u is an odd number of values)."""
+    torch = env["torch"]
+    g = rng(100 * n + m)
+    A, B, C = (g.standard_normal((m, n)) / np.sqrt(n) for _ in range(3))
+    for E in (1, 3, 4001):
+        u = g.uniform(-1, 1, (E, n, n, n))
+        want = env["oracle"].tpo_apply(A, B, C, u)
+        v = torch.full((E, m, m, m), float("nan"), dtype=torch.float64, device=env["dev"])
+        got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C, u)), out=v)
+        torch.cuda.synchronize()
+        assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64, E
+    E = 77
+    u = g.uniform(-1, 1, (E, n, n, n))
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    buf = torch.zeros(u.size + 1, dtype=torch.float64, device=env["dev"])
+    uu = buf[1:].view(u.shape)
+    uu.copy_(to_dev(env, u))
+    got = env["ops"].ekl_tpo_apply(*(to_dev(env, x) for x in (A, B, C)), uu)
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+    A32, B32, C32, u32 = (x.astype(np.float32) for x in (A, B, C, u))
+    want32 = env["oracle"].tpo_apply(A32, B32, C32, u32)
+    got32 = env["ops"].ekl_tpo_apply_f32(*(to_dev(env, x) for x in (A32, B32, C32, u32)))
+    err = env["oracle"].rel_err_per_element(got32.cpu().numpy().astype(np.float64), want32)
+    assert err.max() <= TOL32
+    assert env["ops"].library().ekl_tpo_device_error_flags() == 0
+
+
 @pytest.mark.parametrize("nn,mm", SHAPES[:3])
 def test_apply_f32(env, nn, mm):
     g = rng(3)

@@ -110,10 +110,11 @@ ekl_tpo_status ekl_tpo_inv_helmholtz_lambda(const double* S, const double* lam, 
  *
  * fp64.  With S0 = S1 = S2 it equals ekl_tpo_inv_helmholtz.  v == u exactly (in place) is
  * allowed; any other overlap of v with an input is rejected.  Extents are limited by shared
- * memory (three matrices and two copies of an element).  The cubic shapes 8, 10, 12, 14, 16
- * and the shapes (8,10,12), (12,10,8), (14,12,8), (8,8,16), (16,8,8), with a 16-byte aligned
- * u, run on the FP64 tensor path; every other accepted shape runs on a general kernel with
- * the same results to rounding.
+ * memory (three matrices and two copies of an element).  The cubic shapes with n = 4, 5, 6,
+ * 7, 8, 9, 10, 11, 12, 13, 14, 15, 16 and the shapes (8,10,12), (12,10,8), (14,12,8), (8,8,16),
+ * (16,8,8), (5,7,9), (9,7,5), (6,7,8), (7,8,9) run on the FP64 tensor path (u 16-byte aligned
+ * where n1*n2 is even); every other accepted shape runs on a general kernel with the same
+ * results to rounding.
  */
 ekl_tpo_status ekl_tpo_inv_helmholtz3(const double* S0, const double* S1, const double* S2,
                                       const double* D, const double* u, double* v,

@@ -81,6 +81,7 @@ bool try_launch_convection_odd(const double* Dvq, const double* Ivq, const doubl
 int convection_timeout_flag();
 int convection_odd_timeout_flag();
 int ih3_timeout_flag();
+int ih3_odd_timeout_flag();
 int apply_aniso_timeout_flag();
 int apply_odd_a_timeout_flag();
 int apply_odd_b_timeout_flag();
@@ -109,10 +110,15 @@ bool try_launch_ih_lambda_dmma(const double* S, const double* lam, const double*
 bool try_launch_ih3_dmma(const double* S0, const double* S1, const double* S2, const double* D,
                          const double* u, double* v, int n0, int n1, int n2, long long E,
                          cudaStream_t stream, cudaError_t* err);
-// Forward operator, shapes that are not cubic (fp64).
-bool try_launch_apply_aniso(const double* A, const double* B, const double* C, const double* u,
-                            double* v, int n0, int n1, int n2, int m0, int m1, int m2, long long E,
-                            cudaStream_t stream, cudaError_t* err);
+// The instances of that with an odd extent (their own translation unit).
+bool try_launch_ih3_odd(const double* S0, const double* S1, const double* S2, const double* D,
+                        const double* u, double* v, int n0, int n1, int n2, long long E,
+                        cudaStream_t stream, cudaError_t* err);
+// Forward operator, shapes that are not cubic.
+template <typename T>
+bool try_launch_apply_aniso(const T* A, const T* B, const T* C, const T* u, T* v, int n0, int n1,
+                            int n2, int m0, int m1, int m2, long long E, cudaStream_t stream,
+                            cudaError_t* err);
 // Forward operator, cubic n -> m with an odd extent (three groups of instances, one translation
 // unit each).
 template <typename T>

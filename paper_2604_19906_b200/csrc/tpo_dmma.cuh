@@ -671,11 +671,13 @@ struct Ih3Cfg {
     static constexpr int kByWarps = 20 / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
-    static_assert(N0 % 2 == 0 && N1 % 2 == 0 && N2 % 2 == 0 && N0 >= 4 && N1 >= 4 && N2 >= 4,
-                  "even extents from 4 (bulk copies work in 16-byte units)");
+    // bulk copies need planes that are whole 16-byte units; odd planes use 8-byte asynchronous copies
+    static constexpr bool kBulk = (N1 * N2) % 2 == 0;
+    static_assert(N0 >= 4 && N1 >= 4 && N2 >= 4, "extents from 4 (one tensor step)");
 };
 
-// v[e] = (S0(x)S1(x)S2)(D[e] o ((S0^T(x)S1^T(x)S2^T) u[e])), fp64, u 16-byte aligned.  The
+// v[e] = (S0(x)S1(x)S2)(D[e] o ((S0^T(x)S1^T(x)S2^T) u[e])), fp64, u 16-byte aligned where a
+// plane of u is an even number of values.  The
 // operator fragments of a stage are fetched while the stage before it runs, so that two sets
 // are live at a time whatever the number of distinct matrices.
 template <int N0, int N1, int N2>
@@ -709,9 +711,19 @@ inv_helmholtz3_dmma(const double* __restrict__ S0, const double* __restrict__ S1
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
-    if (q.batch < n_batches && threadIdx.x == 0)
-        load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufA, u + q.batch * C::kBe * kN3,
-                                                     batch_count(q.batch), bar);
+    auto fetch = [&](long long b) {
+        if constexpr (C::kBulk) {
+            if (threadIdx.x == 0) {
+                fence_async_proxy();
+                load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufA, u + b * C::kBe * kN3,
+                                                             batch_count(b), bar);
+            }
+        } else {
+            copy_elements<N0, N1 * N2, C::kPS0, C::kES0, T>(bufA, u + b * C::kBe * kN3,
+                                                            batch_count(b));
+        }
+    };
+    if (q.batch < n_batches) fetch(q.batch);
     OpFrag<F1> f1;
     OpFrag<F2> f2;
     OpFrag<F3> f3;
@@ -731,8 +743,12 @@ inv_helmholtz3_dmma(const double* __restrict__ S0, const double* __restrict__ S1
             bulk_prefetch_l2(u + next * C::kBe * kN3, nbytes);
             bulk_prefetch_l2(D + next * C::kBe * kN3, nbytes);
         }
-        if (!wait_bulk(bar, parity)) break;
-        parity ^= 1u;
+        if constexpr (C::kBulk) {
+            if (!wait_bulk(bar, parity)) break;
+            parity ^= 1u;
+        } else {
+            wait_copies();
+        }
         // forward: S0^T on the slowest axis, then S1^T, then S2^T
         load_op<F2, T>(f2, S1, false, lane);
         run_stage<F1, 0, T, NoFactor, 1>(bufA, bufB, nullptr, f1, none1, none, cnt * F1::kP, warp, lane);
@@ -752,11 +768,7 @@ inv_helmholtz3_dmma(const double* __restrict__ S0, const double* __restrict__ S1
         run_stage<F2, 0, T, NoFactor, 1>(bufA, bufB, nullptr, f2, none2, none, cnt * F2::kP, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
-        if (next < n_batches && threadIdx.x == 0) {
-            fence_async_proxy();
-            load_elements<N0, N1 * N2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
-                                                         batch_count(next), bar);
-        }
+        if (next < n_batches) fetch(next);
         load_op<F1, T>(f1, S0, false, lane);
         run_stage<B3, 2, T, NoFactor, 1>(bufB, nullptr, v + e0 * kN3, f3, dfac, none, cnt * B3::kP, warp, lane);
         q.publish();

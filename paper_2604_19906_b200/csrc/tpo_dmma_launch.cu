@@ -259,16 +259,8 @@ bool try_launch_apply_dmma(const T* A, const T* B, const T* C, const T* u, T* v,
     // fp64 u is bulk-copied plane by plane where a plane is a whole number of 16-byte units:
     // 16-byte aligned element addresses
     if (sizeof(T) == 8 && (n1 * n2) % 2 == 0 && reinterpret_cast<uintptr_t>(u) % 16) return false;
-    if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2) {
-        if constexpr (sizeof(T) == 8)
-            return try_launch_apply_aniso(reinterpret_cast<const double*>(A),
-                                          reinterpret_cast<const double*>(B),
-                                          reinterpret_cast<const double*>(C),
-                                          reinterpret_cast<const double*>(u),
-                                          reinterpret_cast<double*>(v), n0, n1, n2, m0, m1, m2, E,
-                                          stream, err);
-        return false;
-    }
+    if (n0 != n1 || n1 != n2 || m0 != m1 || m1 != m2)
+        return try_launch_apply_aniso(A, B, C, u, v, n0, n1, n2, m0, m1, m2, E, stream, err);
     if (try_launch_apply_tf32(A, B, C, u, v, n0, m0, E, stream, err)) return true;
     switch (n0) {
         case 4: if (apply_cubic_from<4, T>(m0, A, B, C, u, v, E, stream, err)) return true; break;
@@ -331,7 +323,8 @@ extern "C" int ekl_tpo_device_error_flags(void) {
     const int flags[] = {ekl::dmma::take_timeout_flag(),   ekl::convection_timeout_flag(),
                          ekl::ih3_timeout_flag(),          ekl::apply_aniso_timeout_flag(),
                          ekl::apply_odd_a_timeout_flag(),  ekl::apply_odd_b_timeout_flag(),
-                         ekl::apply_odd_c_timeout_flag(),    ekl::convection_odd_timeout_flag()};
+                         ekl::apply_odd_c_timeout_flag(),    ekl::convection_odd_timeout_flag(),
+                         ekl::ih3_odd_timeout_flag()};
     int all = 0;
     for (int f : flags) {
         if (f < 0) return -1;

@@ -7,9 +7,12 @@ pytestmark = pytest.mark.gpu
 
 TOL64 = 1e-12
 # shapes with a tensor-path instance, then shapes that take the general kernel
-TENSOR_SHAPES = [(8, 8, 8), (10, 10, 10), (12, 12, 12), (14, 14, 14), (16, 16, 16),
-                 (8, 10, 12), (12, 10, 8), (14, 12, 8), (8, 8, 16), (16, 8, 8)]
-GENERAL_SHAPES = [(1, 1, 1), (2, 3, 4), (5, 4, 3), (7, 7, 7), (6, 8, 10), (9, 2, 11),
+TENSOR_SHAPES = [(4, 4, 4), (6, 6, 6), (8, 8, 8), (10, 10, 10), (12, 12, 12), (14, 14, 14),
+                 (16, 16, 16), (8, 10, 12), (12, 10, 8), (14, 12, 8), (8, 8, 16), (16, 8, 8),
+                 # with an odd extent: u comes in by 8-byte copies where a plane is odd
+                 (5, 5, 5), (7, 7, 7), (9, 9, 9), (11, 11, 11), (13, 13, 13), (15, 15, 15),
+                 (5, 7, 9), (9, 7, 5), (6, 7, 8), (7, 8, 9)]
+GENERAL_SHAPES = [(1, 1, 1), (2, 3, 4), (5, 4, 3), (7, 7, 5), (6, 8, 10), (9, 2, 11),
                   (13, 14, 15), (18, 4, 4), (1, 16, 3)]
 
 
@@ -51,7 +54,8 @@ def test_matches_oracle(env, nn, E):
     assert err.max() <= TOL64, (nn, E, err.max())
 
 
-@pytest.mark.parametrize("nn", [(14, 14, 14), (8, 10, 12), (16, 8, 8), (5, 4, 3)])
+@pytest.mark.parametrize("nn", [(14, 14, 14), (8, 10, 12), (16, 8, 8), (5, 4, 3), (9, 9, 9), (5, 7, 9),
+                                (6, 7, 8)])
 def test_many_batches_per_cta_in_place_and_repeatable(env, nn):
     """Enough elements that every CTA draws several batches; in place; bitwise repeatable."""
     torch = env["torch"]
@@ -67,6 +71,13 @@ def test_many_batches_per_cta_in_place_and_repeatable(env, nn):
     torch.cuda.synchronize()
     assert env["oracle"].rel_err_per_element(a.cpu().numpy(), want).max() <= TOL64
     assert torch.equal(a, b) and torch.equal(a, inplace)
+    if (nn[1] * nn[2]) % 2 == 1:
+        # odd planes: u may start 8 bytes off a 16-byte boundary and still take the same kernel
+        buf = torch.zeros(ud.numel() + 1, dtype=torch.float64, device=env["dev"])
+        shifted = buf[1:].view(ud.shape)
+        shifted.copy_(ud)
+        c = env["ops"].ekl_tpo_inv_helmholtz3(*Sd, Dd, shifted)
+        assert torch.equal(a, c)
     assert env["ops"].library().ekl_tpo_device_error_flags() == 0
 
 

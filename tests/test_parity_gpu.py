@@ -306,6 +306,20 @@ def test_apply_f64_non_cubic_shapes_on_the_tensor_path(env, nn, mm, E):
         assert env["oracle"].rel_err_per_element(got2.cpu().numpy(), want).max() <= TOL64
 
 
+@pytest.mark.parametrize("nn,mm", ANISO)
+def test_apply_f32_non_cubic_shapes(env, nn, mm):
+    """The non-cubic tensor-path shapes with fp32 fields (widened on chip, fp64 arithmetic)."""
+    g = rng(hash((mm, nn)) % 9973)
+    E = 203
+    A, B, C = ((g.standard_normal((mm[d], nn[d])) / np.sqrt(nn[d])).astype(np.float32)
+               for d in range(3))
+    u = g.uniform(-1, 1, (E,) + nn).astype(np.float32)
+    want = env["oracle"].tpo_apply(A, B, C, u)
+    got = env["ops"].ekl_tpo_apply_f32(*(to_dev(env, x) for x in (A, B, C, u)))
+    err = env["oracle"].rel_err_per_element(got.cpu().numpy().astype(np.float64), want)
+    assert err.max() <= TOL32
+
+
 ODD_CUBIC = [(5, 5), (7, 7), (9, 9), (11, 11), (13, 13), (15, 15), (5, 7), (7, 5), (7, 9), (9, 7),
              (9, 11), (11, 9), (11, 13), (13, 11), (13, 15), (15, 13), (5, 8), (8, 5), (6, 9), (9, 6),
              (7, 11), (11, 7), (9, 14), (14, 9), (10, 15), (15, 10), (4, 5), (5, 4), (5, 6), (6, 5),

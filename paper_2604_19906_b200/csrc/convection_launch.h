@@ -12,16 +12,16 @@ cudaError_t launch_conv(const double* Dvq, const double* Ivq, const double* M, c
                         double* F, long long E, cudaStream_t stream) {
     using C = dmma::ConvCfg<NQ, NV>;
     static_assert(C::kSmemBytes <= kMaxSmemBytes, "instance does not fit in shared memory");
-    static bool prepared[64] = {false};
+    static std::atomic<int> prepared[64];   // racing first calls store the same value
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!prepared[dev]) {
+    if (!prepared[dev].load(std::memory_order_acquire)) {
         err = cudaFuncSetAttribute(dmma::convection_dmma<NQ, NV>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
         if (err != cudaSuccess) return err;
-        prepared[dev] = true;
+        prepared[dev].store(1, std::memory_order_release);
     }
     long long grid = (long long)sm_count() * C::kCtasPerSm;
     if (grid > E) grid = E;

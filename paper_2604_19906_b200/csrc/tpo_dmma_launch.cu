@@ -65,16 +65,16 @@ template <int N>
 cudaError_t launch_ih_umma(const float* S, const float* D, const float* u, float* v, long long E,
                            cudaStream_t stream) {
     using C = umma::Cfg<N>;
-    static bool ready[64] = {false};
+    static std::atomic<int> ready[64];   // racing first calls store the same value
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!ready[dev]) {
+    if (!ready[dev].load(std::memory_order_acquire)) {
         err = cudaFuncSetAttribute(umma::inv_helmholtz_umma<N>,
                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
         if (err != cudaSuccess) return err;
-        ready[dev] = true;
+        ready[dev].store(1, std::memory_order_release);
     }
     // as many CTAs as shared memory lets an SM hold (the occupancy query answers 1 for kernels
     // that allocate tensor memory; more do run side by side, 32 columns each)

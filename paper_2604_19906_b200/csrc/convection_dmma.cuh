@@ -134,7 +134,6 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
     if (threadIdx.x == 0) mbar_init(bar, 1);
     __syncthreads();
 
-    // thread 0: bulk-copy the P fields of (c, e) -- and M[e] when asked -- plane by plane
     auto fetch = [&](int c, long long e, bool with_m) {
         const unsigned field = (unsigned)(kQ3 * sizeof(double));
         mbar_expect_tx(bar, (with_m ? 4u : 3u) * field);
@@ -175,6 +174,9 @@ convection_dmma(const double* __restrict__ Dvq, const double* __restrict__ Ivq,
             const unsigned field = (unsigned)(kQ3 * sizeof(double));
             for (int cd = 3; cd < 9; ++cd) bulk_prefetch_l2(P + ((size_t)cd * E + e) * kQ3, field);
         }
+        // (unrolled: the compiler does not do it by itself with the early exit in the loop, and
+        // the rolled loop measured 8 % slower)
+#pragma unroll
         for (int c = 0; c < 3; ++c) {
             if constexpr (C::kBulk) {
                 if (!wait_bulk(bar, parity)) {

@@ -171,18 +171,25 @@ __device__ __forceinline__ void run_stage32(const float* __restrict__ in, float*
     }
 }
 
-// Thread 0: `cnt` dense elements of K planes x P floats each into the plane-padded layout.
-template <int K, int P, int PS, int ES>
+// `cnt` dense elements of K planes x P floats each into the plane-padded layout, all copies
+// completing on `bar`.  Called by thread 0 (LANES = 1) or by the CTA's first warp (LANES = 32,
+// `lane` = threadIdx.x): lane 0 announces the bytes and the lanes issue the per-plane copies side
+// by side -- one thread issuing dozens of copies in a row takes about as long as the copies
+// themselves, which shows where they have little time to land (measured: 3.6 % at n = 14, 1.6 %
+// at n = 16, but 6 % slower at n = 12).  A copy may complete before lane 0 has announced it: the
+// phase cannot end before lane 0's arrival, and by then the byte count balances.
+template <int K, int P, int PS, int ES, int LANES>
 __device__ __forceinline__ void load_elements32(float* dst, const float* src, int cnt,
-                                                uint64_t* bar) {
-    dmma::mbar_expect_tx(bar, (unsigned)(cnt * K * P * sizeof(float)));
+                                                uint64_t* bar, int lane) {
+    if (lane == 0) dmma::mbar_expect_tx(bar, (unsigned)(cnt * K * P * sizeof(float)));
     if (PS == P && ES == K * P) {
-        dmma::bulk_load(dst, src, (unsigned)(cnt * K * P * sizeof(float)), bar);
+        if (lane == 0) dmma::bulk_load(dst, src, (unsigned)(cnt * K * P * sizeof(float)), bar);
     } else {
-        for (int e = 0; e < cnt; ++e)
-            for (int x = 0; x < K; ++x)
-                dmma::bulk_load(dst + e * ES + x * PS, src + (size_t)(e * K + x) * P,
-                                (unsigned)(P * sizeof(float)), bar);
+        for (int i = lane; i < cnt * K; i += LANES) {
+            const int e = i / K, x = i - e * K;
+            dmma::bulk_load(dst + e * ES + x * PS, src + (size_t)i * P,
+                            (unsigned)(P * sizeof(float)), bar);
+        }
     }
 }
 
@@ -196,6 +203,8 @@ struct IhCfg32 {
     static constexpr int kRS = pad_row32(N), kPS = pad_plane32(N * kRS), kES = N * kPS;
     static constexpr int kElemBuf = (kES0 > kES ? kES0 : kES);
     static constexpr int kBe = 2;
+    // threads that issue the bulk copies of u (see load_elements32)
+    static constexpr int kCopyLanes = (N >= 14) ? 32 : 1;
     static constexpr int kTiles = kBe * N * N / 8;
     // an even deal of the tiles; 4 warps (more CTAs per SM) measured 4-6 % faster for n = 8, 12
     static constexpr int kWarps = (N == 8 || N == 12) ? 4
@@ -252,9 +261,9 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
         const long long e0 = b * C::kBe;
         return (int)((E - e0 < C::kBe) ? (E - e0) : C::kBe);
     };
-    if (q.batch < n_batches && threadIdx.x == 0)
-        load_elements32<N, kN2, C::kPS0, C::kES0>(bufA, u + q.batch * C::kBe * kN3,
-                                                  batch_count(q.batch), bar);
+    if (q.batch < n_batches && threadIdx.x < C::kCopyLanes)
+        load_elements32<N, kN2, C::kPS0, C::kES0, C::kCopyLanes>(
+            bufA, u + q.batch * C::kBe * kN3, batch_count(q.batch), bar, threadIdx.x);
     unsigned parity = 0;
     while (q.batch < n_batches) {
         q.draw();
@@ -286,10 +295,10 @@ inv_helmholtz_tf32(const float* __restrict__ S, const float* __restrict__ D, con
         run_stage32<Mid, 0, FD>(bufA, bufB, nullptr, opb, dfac, Db, valid, warp, lane);
         __syncthreads();
         // bufA is free: bring in the next batch while the last stage streams v out
-        if (next < n_batches && threadIdx.x == 0) {
+        if (next < n_batches && threadIdx.x < C::kCopyLanes) {
             dmma::fence_async_proxy();
-            load_elements32<N, kN2, C::kPS0, C::kES0>(bufA, u + next * C::kBe * kN3,
-                                                      batch_count(next), bar);
+            load_elements32<N, kN2, C::kPS0, C::kES0, C::kCopyLanes>(
+                bufA, u + next * C::kBe * kN3, batch_count(next), bar, threadIdx.x);
         }
         run_stage32<Last, 2, FD>(bufB, nullptr, v + e0 * kN3, opb, dfac, Db, valid, warp, lane);
         q.publish();
@@ -372,8 +381,8 @@ apply_tf32(const float* __restrict__ A, const float* __restrict__ B, const float
     auto fetch = [&](long long b) {
         if (threadIdx.x == 0) {
             dmma::fence_async_proxy();
-            load_elements32<N0, N1 * N2, C::kPS0, C::kES0>(bufU, u + b * C::kBe * S1::kIn,
-                                                           batch_count(b), bar);
+            load_elements32<N0, N1 * N2, C::kPS0, C::kES0, 1>(bufU, u + b * C::kBe * S1::kIn,
+                                                              batch_count(b), bar, 0);
         }
     };
     if (q.batch < n_batches) fetch(q.batch);

@@ -22,8 +22,8 @@
  *    validates its arguments on the host, enqueues work on `stream` and returns.
  *    Buffers must stay valid until the stream has passed that work.  Inputs are
  *    only read; the output is fully overwritten.
- *  - Work distribution: a launch in which a CTA gets more than one batch of
- *    elements hands the batches out through a counter (16 bytes) taken from a fixed
+ *  - Work distribution: most kernels, in a launch that gives a CTA more than four
+ *    batches of elements, hand the batches out through a counter (16 bytes) taken from a fixed
  *    ring of 4096 inside the library image.  The kernel itself puts the counter back
  *    to zero when its last CTA leaves, so a call is still one kernel launch and
  *    nothing else.  A counter comes round again after 4096 launches; a kernel whose

@@ -452,3 +452,70 @@ def test_device_input_generators_match_the_host_bit_for_bit(env):
             h = host[key]
             d = dev[key].cpu().numpy() if hasattr(dev[key], "cpu") else dev[key]
             assert np.array_equal(h, d), (idx, key)
+
+
+# --------------------------------------------------------------------------- element independence
+
+@pytest.mark.parametrize("n,dtype", [(14, "f64"), (8, "f64"), (5, "f64"), (3, "f64"), (12, "f64"),
+                                     (14, "f32"), (8, "f32"), (7, "f32")])
+def test_elements_are_independent(env, n, dtype):
+    """The elements of a batch share tensor tiles and shared-memory buffers, but every result
+    depends on its own element only: with NaN and Inf written into a few elements of u and D,
+    every other element of v is bit-identical to the clean run, and the poisoned ones are not
+    finite.  Covers both neighbours in a batch of two, a whole batch, and the last (partly
+    filled) batch."""
+    torch = env["torch"]
+    E = 1203
+    S, D, u = synth_ih(n, E, 31 * n)
+    tdt = torch.float64 if dtype == "f64" else torch.float32
+    fn = env["ops"].ekl_tpo_inv_helmholtz if dtype == "f64" else env["ops"].ekl_tpo_inv_helmholtz_f32
+    Sd, Dd, ud = (to_dev(env, x, tdt) for x in (S, D, u))
+    clean = fn(Sd, Dd, ud).clone()
+    bad_u = [0, 5, 400, 401, E - 1]
+    bad_d = [77, 800]
+    up, Dp = ud.clone(), Dd.clone()
+    for k, e in enumerate(bad_u):
+        up[e].view(-1)[(13 * k) % n ** 3] = float("nan") if k % 2 == 0 else float("inf")
+    for e in bad_d:
+        Dp[e].view(-1)[n ** 3 - 1] = float("nan")
+    got = fn(Sd, Dp, up)
+    torch.cuda.synchronize()
+    bad = torch.zeros(E, dtype=torch.bool, device=env["dev"])
+    bad[bad_u + bad_d] = True
+    assert torch.equal(got[~bad], clean[~bad])
+    assert not bool(torch.isfinite(got[bad]).all(dim=(1, 2, 3)).any())
+
+
+def test_forward_and_convection_elements_are_independent(env):
+    torch = env["torch"]
+    g = rng(99)
+    E = 777
+    A, B, C = (g.standard_normal((12, 8)) / 3 for _ in range(3))
+    u = g.uniform(-1, 1, (E, 8, 8, 8))
+    dev = [to_dev(env, x) for x in (A, B, C, u)]
+    clean = env["ops"].ekl_tpo_apply(*dev).clone()
+    up = dev[3].clone()
+    for e in (1, 300, E - 1):
+        up[e, 3, 4, 5] = float("nan")
+    got = env["ops"].ekl_tpo_apply(dev[0], dev[1], dev[2], up)
+    bad = torch.zeros(E, dtype=torch.bool, device=env["dev"])
+    bad[[1, 300, E - 1]] = True
+    assert torch.equal(got[~bad], clean[~bad])
+    assert bool(torch.isnan(got[bad]).any(dim=(1, 2, 3)).all())
+    # convection: a NaN in M[e] reaches all three components of element e and nothing else
+    nq, nv, Ec = 12, 8, 333
+    Dvq, Ivq = (to_dev(env, g.standard_normal((nv, nq)) / 3) for _ in range(2))
+    M = to_dev(env, g.uniform(0.5, 1.5, (Ec, nq, nq, nq)))
+    P = to_dev(env, g.uniform(-1, 1, (3, 3, Ec, nq, nq, nq)))
+    clean = env["ops"].ekl_tpo_convection(Dvq, Ivq, M, P).clone()
+    Mp = M.clone()
+    Mp[100, 0, 0, 0] = float("nan")
+    Pp = P.clone()
+    Pp[1, 2, 200, 5, 5, 5] = float("inf")
+    got = env["ops"].ekl_tpo_convection(Dvq, Ivq, Mp, Pp)
+    torch.cuda.synchronize()
+    same = torch.ones(3, Ec, dtype=torch.bool, device=env["dev"])
+    same[:, 100] = False
+    same[1, 200] = False
+    assert torch.equal(got[same], clean[same])
+    assert not bool(torch.isfinite(got[~same]).all(dim=(1, 2, 3)).any())

@@ -399,3 +399,35 @@ def test_rel_err_per_element_edge_cases():
     v[2, 1] = np.inf
     assert oracle.rel_err_per_element(v, ref)[2] == np.inf
     assert np.array_equal(oracle.rel_err_per_element(ref, ref), np.zeros(3))
+
+
+def test_scaling_by_a_power_of_two_is_exact_in_every_oracle_routine():
+    """Each routine is linear in its field arguments, and a power of two changes no rounding:
+    scaling u (or D, M, P) by 2^k scales the result by 2^k bit for bit.  A routine that took a
+    square root, normalised, or mixed its arguments non-linearly would fail."""
+    g = np.random.Generator(np.random.PCG64(2024))
+    f = 2.0 ** 37
+    n, E = 5, 3
+    S = g.standard_normal((n, n))
+    D = g.uniform(0.1, 1.0, (E, n, n, n))
+    u = g.standard_normal((E, n, n, n))
+    base = oracle.inv_helmholtz(S, D, u)
+    assert np.array_equal(oracle.inv_helmholtz(S, D, u * f), base * f)
+    assert np.array_equal(oracle.inv_helmholtz(S, D * f, u), base * f)
+    nn = (3, 4, 5)
+    S3 = [g.standard_normal((k, k)) for k in nn]
+    D3 = g.uniform(0.1, 1.0, (E,) + nn)
+    u3 = g.standard_normal((E,) + nn)
+    base3 = oracle.inv_helmholtz3(*S3, D3, u3)
+    assert np.array_equal(oracle.inv_helmholtz3(*S3, D3 / f, u3), base3 / f)
+    assert np.array_equal(oracle.inv_helmholtz3(*S3, D3, u3 * f), base3 * f)
+    A, B, C = g.standard_normal((4, 3)), g.standard_normal((2, 4)), g.standard_normal((6, 5))
+    ua = g.standard_normal((E, 3, 4, 5))
+    assert np.array_equal(oracle.tpo_apply(A, B, C, ua * f), oracle.tpo_apply(A, B, C, ua) * f)
+    nq, nv = 4, 3
+    Dvq, Ivq = g.standard_normal((nv, nq)), g.standard_normal((nv, nq))
+    M = g.uniform(0.5, 1.5, (E, nq, nq, nq))
+    P = g.standard_normal((3, 3, E, nq, nq, nq))
+    basec = oracle.convection(Dvq, Ivq, M, P)
+    assert np.array_equal(oracle.convection(Dvq, Ivq, M * f, P), basec * f)
+    assert np.array_equal(oracle.convection(Dvq, Ivq, M, P / f), basec / f)

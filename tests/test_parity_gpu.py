@@ -519,3 +519,24 @@ def test_forward_and_convection_elements_are_independent(env):
     same[1, 200] = False
     assert torch.equal(got[same], clean[same])
     assert not bool(torch.isfinite(got[~same]).all(dim=(1, 2, 3)).any())
+
+
+@pytest.mark.parametrize("n,dtype,k", [(14, "f64", 400), (14, "f64", -400), (9, "f64", 300),
+                                       (3, "f64", -300), (14, "f32", 40), (12, "f32", -40),
+                                       (7, "f32", 30)])
+def test_scaling_by_a_power_of_two_is_exact(env, n, dtype, k):
+    """The operator is linear in u and in D, and a power of two changes no rounding while
+    nothing overflows or underflows: v(2^k u, D) = v(u, 2^k D) = 2^k v(u, D) bit for bit.
+    A hidden conversion to a narrower format (or a fused multiply that is not there in the
+    other run) would break it; so would the split of fp32 values into TF32 parts if it were
+    not scale invariant."""
+    torch = env["torch"]
+    E = 129
+    S, D, u = synth_ih(n, E, 17 * n + 3)
+    tdt = torch.float64 if dtype == "f64" else torch.float32
+    fn = env["ops"].ekl_tpo_inv_helmholtz if dtype == "f64" else env["ops"].ekl_tpo_inv_helmholtz_f32
+    Sd, Dd, ud = (to_dev(env, x, tdt) for x in (S, D, u))
+    base = fn(Sd, Dd, ud)
+    f = 2.0 ** k
+    assert torch.equal(fn(Sd, Dd, ud * f), base * f)
+    assert torch.equal(fn(Sd, Dd * f, ud), base * f)

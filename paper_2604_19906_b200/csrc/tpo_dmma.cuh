@@ -481,9 +481,10 @@ struct IhCfg {
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
     // warps per CTA: an even deal of the tiles where one exists, with the measured exceptions
     // (CTAs of 5 warps load the four scheduler partitions 2,1,1,1: n = 10 and 20 run 8 % and
-    // 26 % faster with 4 and 8 warps, n = 17 12 % faster with 4)
+    // 26 % faster with 4 and 8 warps, n = 17 12 % faster with 4; n = 7 and 9 1 % and 4 % faster
+    // with 4)
     static constexpr int kWarps = (N == 14 || N == 20) ? 8
-                                  : (N == 10 || N == 17) ? 4
+                                  : (N == 7 || N == 9 || N == 10 || N == 17) ? 4
                                   : (kTiles <= 36 && kTiles % 4 == 0) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6

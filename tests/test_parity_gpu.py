@@ -540,3 +540,21 @@ def test_scaling_by_a_power_of_two_is_exact(env, n, dtype, k):
     f = 2.0 ** k
     assert torch.equal(fn(Sd, Dd, ud * f), base * f)
     assert torch.equal(fn(Sd, Dd * f, ud), base * f)
+
+
+@pytest.mark.parametrize("n,E", [(5, 4099), (7, 3001), (9, 2501), (11, 1801), (13, 1201), (5, 6), (9, 4)])
+def test_inv_helmholtz_odd_n_aligned_fields_many_batches(env, n, E):
+    """Odd n with 16-byte aligned fields (the other odd-n cases offset them by 8 bytes), an odd E
+    that leaves a partly filled last batch, several batches per CTA; also in place."""
+    torch = env["torch"]
+    S, D, u = synth_ih(n, E, 9100 + n)
+    want = env["oracle"].inv_helmholtz(S, D, u)
+    Sd, Dd, ud = to_dev(env, S), to_dev(env, D), to_dev(env, u)
+    assert ud.data_ptr() % 16 == 0
+    got = env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, ud)
+    env["torch"].cuda.synchronize()
+    assert env["oracle"].rel_err_per_element(got.cpu().numpy(), want).max() <= TOL64
+    inplace = ud.clone()
+    env["ops"].ekl_tpo_inv_helmholtz(Sd, Dd, inplace, out=inplace)
+    assert torch.equal(inplace, got)
+    assert env["ops"].library().ekl_tpo_device_error_flags() == 0

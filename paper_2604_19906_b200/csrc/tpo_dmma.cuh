@@ -476,15 +476,18 @@ struct IhCfg {
     // layout between stages
     static constexpr int kRS = pad_row(N), kPS = pad_plane(N * kRS), kES = N * kPS;
     static constexpr int kElemBuf = (kES0 > kES ? kES0 : kES);
-    // elements per batch: two (four for the smallest) unless that leaves room for one CTA only
-    static constexpr int kBe = (N <= 6) ? 4 : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
+    // elements per batch: two (four for the smallest) unless that leaves room for one CTA only;
+    // n = 11 and 12 measured 9 % and 2-3 % faster with one element and more, smaller CTAs
+    static constexpr int kBe = (N <= 6) ? 4
+                               : (N == 11 || N == 12) ? 1
+                               : ((4 * kElemBuf * 8 <= 112 * 1024) ? 2 : 1);
     static constexpr int kTiles = (kBe * N * N + 7) / 8;
     // warps per CTA: an even deal of the tiles where one exists, with the measured exceptions
     // (CTAs of 5 warps load the four scheduler partitions 2,1,1,1: n = 10 and 20 run 8 % and
     // 26 % faster with 4 and 8 warps, n = 17 12 % faster with 4; n = 7 and 9 1 % and 4 % faster
-    // with 4)
-    static constexpr int kWarps = (N == 14 || N == 20) ? 8
-                                  : (N == 7 || N == 9 || N == 10 || N == 17) ? 4
+    // with 4; n = 16 4 % faster with three CTAs of 8 than of 4)
+    static constexpr int kWarps = (N == 14 || N == 16 || N == 20) ? 8
+                                  : (N == 7 || N == 9 || N == 10 || N == 11 || N == 12 || N == 17) ? 4
                                   : (kTiles <= 36 && kTiles % 4 == 0) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6
@@ -503,7 +506,8 @@ struct IhCfg {
     static constexpr size_t kSmemBytes =
         2 * (size_t)kBufElems * sizeof(double) + kStagingBytes + 16;
     static constexpr int kBySmem = (int)((227 * 1024) / (kSmemBytes + 1024));
-    static constexpr int kByWarps = 20 / kWarps;
+    // at most 20 warps per SM; 24 for n = 16, where a third CTA of 8 warps fits (4 % faster)
+    static constexpr int kByWarps = (N == 16 ? 24 : 20) / kWarps;
     static constexpr int kCtasPerSm =
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
     // bulk copies need 16-byte granules: even N; odd N uses 8-byte asynchronous copies

@@ -202,12 +202,15 @@ struct IhCfg32 {
     static constexpr int kPS0 = pad_plane32(N * N), kES0 = N * kPS0;
     static constexpr int kRS = pad_row32(N), kPS = pad_plane32(N * kRS), kES = N * kPS;
     static constexpr int kElemBuf = (kES0 > kES ? kES0 : kES);
-    static constexpr int kBe = 2;
+    // one element per batch in more, smaller CTAs measured 5 % (n = 8), 7 % (12), 5 % (14) and
+    // 10 % (16) faster than two; n = 10 is 5 % faster with two
+    static constexpr int kBe = (N == 10) ? 2 : 1;
     // threads that issue the bulk copies of u (see load_elements32)
     static constexpr int kCopyLanes = (N >= 14) ? 32 : 1;
-    static constexpr int kTiles = kBe * N * N / 8;
-    // an even deal of the tiles; 4 warps (more CTAs per SM) measured 4-6 % faster for n = 8, 12
-    static constexpr int kWarps = (N == 8 || N == 12) ? 4
+    static constexpr int kTiles = (kBe * N * N + 7) / 8;
+    // an even deal of the tiles; 4 warps (more CTAs per SM) measured 4-6 % faster for n = 8, 12,
+    // and for n = 14 (25 tiles) faster than 5, 6 or 8
+    static constexpr int kWarps = (N == 8 || N == 12 || N == 14) ? 4
                                   : (kTiles % 8 == 0) ? 8
                                   : (kTiles % 6 == 0) ? 6
                                   : (kTiles % 5 == 0) ? 5

@@ -135,11 +135,8 @@ cudaError_t launch_ap_tf32(const float* A, const float* B, const float* Cm, cons
     long long grid = (long long)sm_count() * per_sm;
     if (grid > batches) grid = batches;
     unsigned long long* tickets = nullptr;
-    // (from 16 points the fixed deal measured faster: 16 -> 16 by 8 %, 16 -> 12 by 3 %)
-    if (N < 16) {
-        err = tickets_for(batches, grid, &tickets);
-        if (err != cudaSuccess) return err;
-    }
+    err = tickets_for(batches, grid, &tickets);
+    if (err != cudaSuccess) return err;
     kernel<<<(unsigned)grid, C::kThreads, C::kSmemBytes, stream>>>(A, B, Cm, u, v, E, tickets);
     return cudaGetLastError();
 }

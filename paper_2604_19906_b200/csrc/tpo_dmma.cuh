@@ -793,8 +793,13 @@ struct ApplyCfg {
     static constexpr int kRS1 = pad_row(M0), kPS1 = pad_plane(N2 * kRS1), kES1 = N1 * kPS1;
     // after the second stage: [n2][m0][m1]
     static constexpr int kRS2 = pad_row(M1), kPS2 = pad_plane(M0 * kRS2), kES2 = N2 * kPS2;
-    // two elements per batch unless that leaves room for one CTA per SM only
-    static constexpr int kBe = ((kES0 + kES1 + kES2) * 2 * 8 <= 112 * 1024) ? 2 : 1;
+    // two elements per batch for inputs of up to 8 points in the first direction, and for 10; one
+    // otherwise (more, smaller CTAs).  Measured with one instead of two: 12 -> 8 15 %, 12 -> 12 7 %,
+    // 9 -> 9 17 %, 11 -> 11 24 %, 13 -> 13 14 %, 7 -> 11 32 % faster; 8 -> 12 9 %, 8 -> 8 5 %,
+    // 6 -> 10 19 %, 10 -> 10 7 %, 10 -> 14 7 %, 7 -> 7 13 % slower
+    static constexpr bool kSmallInput = (N0 <= 8 || N0 == 10) && !(N0 == 7 && M0 > 8);
+    static constexpr int kBe =
+        ((kES0 + kES1 + kES2) * 2 * 8 <= 112 * 1024 && kSmallInput) ? 2 : 1;
     // the last stage has the most tiles; give every warp at most about a dozen
     static constexpr int kWarps = (kBe * M0 * M1 / 8 > 48) ? 8 : 4;
     using S1 = Stage<N0, M0, N1, N2, kBe, kWarps, N2, kPS0, kES0, kRS1, kPS1, kES1>;

@@ -227,7 +227,8 @@ struct IhCfg32 {
         (kBySmem < kByWarps ? kBySmem : kByWarps) < 1 ? 1 : (kBySmem < kByWarps ? kBySmem : kByWarps);
     // tiles of the pointwise factor held ahead in registers: deeper than this spills at the
     // 80 registers three CTAs per SM leave a thread (measured: n = 14 9 % and n = 8 12 % faster)
-    static constexpr int kFactorDepth = (N == 8) ? 1 : 2;
+    // (n = 14, seven tiles per warp and stage: three ahead is another 2 % faster)
+    static constexpr int kFactorDepth = (N == 8) ? 1 : (N == 14) ? 3 : 2;
 };
 
 // v[e] = (S(x)S(x)S)(D[e] o ((S^T(x)S^T(x)S^T) u[e])), fp32 fields; u must be 16-byte aligned.
